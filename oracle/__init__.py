@@ -1,0 +1,179 @@
+"""CPU oracle of the Orthrus generation-step hot path: TEST INFRASTRUCTURE ONLY.
+
+A thin ctypes loader around `orthrus_oracle.c` (plain C, fp64 accumulation).
+Only the test suite, the smoke check and the benchmark's CPU-baseline leg may
+import this package; the CUDA library and its Python binding never do.
+
+All tensors are torch CPU tensors (bf16, fp32 or fp64, contiguous).  Attention
+results come back as float64 tensors.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "orthrus_oracle.c")
+_LIB = os.path.join(_HERE, "liborthrus_oracle.so")
+
+VIEW_DIFFUSION = 0
+VIEW_AR = 1
+
+_DTYPE_CODE = {torch.bfloat16: 0, torch.float32: 1, torch.float64: 2}
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, OpenMP) next to its source."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + f".tmp{os.getpid()}"
+    subprocess.run(["gcc", "-O2", "-fopenmp", "-std=c11", "-shared", "-fPIC",
+                    "-o", tmp, _SRC, "-lm"], check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _AttnDesc(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("block", ctypes.c_int32),
+                ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("capacity", ctypes.c_int64),
+                ("q", ctypes.c_void_p), ("k_blk", ctypes.c_void_p),
+                ("v_blk", ctypes.c_void_p), ("k_cache", ctypes.c_void_p),
+                ("v_cache", ctypes.c_void_p), ("cache_len", ctypes.c_void_p),
+                ("scale", ctypes.c_double)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_block_attend.restype = ctypes.c_int
+        _lib.oracle_block_attend.argtypes = [ctypes.POINTER(_AttnDesc), ctypes.c_int,
+                                             ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64]
+        _lib.oracle_block_attend_rows.restype = ctypes.c_int
+        _lib.oracle_block_attend_rows.argtypes = [ctypes.POINTER(_AttnDesc), ctypes.c_int,
+                                                  ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]
+        _lib.oracle_consensus_accept.restype = ctypes.c_int
+        _lib.oracle_consensus_accept.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p,
+                                                 ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                                 ctypes.c_void_p, ctypes.c_void_p,
+                                                 ctypes.c_void_p, ctypes.c_void_p]
+        _lib.oracle_kv_append.restype = ctypes.c_int
+        _lib.oracle_kv_append.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                          ctypes.c_int32, ctypes.c_int64, ctypes.c_int,
+                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.c_int]
+        _lib.oracle_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def _check(t: torch.Tensor, name: str) -> torch.Tensor:
+    if t.device.type != "cpu" or not t.is_contiguous():
+        raise ValueError(f"{name}: the oracle takes contiguous CPU tensors")
+    return t
+
+
+def _desc(q, k_blk, v_blk, k_cache, v_cache, cache_len, scale) -> _AttnDesc:
+    B, K, Hq, d = q.shape
+    Hkv, cap = k_cache.shape[1], k_cache.shape[2]
+    dt = q.dtype
+    for n, t in (("q", q), ("k_blk", k_blk), ("v_blk", v_blk),
+                 ("k_cache", k_cache), ("v_cache", v_cache)):
+        _check(t, n)
+        if t.dtype != dt:
+            raise ValueError("all attention tensors must share one dtype")
+    if tuple(k_blk.shape) != (B, K, Hkv, d) or tuple(v_blk.shape) != (B, K, Hkv, d):
+        raise ValueError("block KV must be [B][K][Hkv][d]")
+    if tuple(k_cache.shape) != (B, Hkv, cap, d) or tuple(v_cache.shape) != (B, Hkv, cap, d):
+        raise ValueError("cache must be [B][Hkv][capacity][d]")
+    _check(cache_len, "cache_len")
+    if cache_len.dtype != torch.int32 or cache_len.numel() != B:
+        raise ValueError("cache_len must be int32 [B]")
+    return _AttnDesc(B, K, Hq, Hkv, d, _DTYPE_CODE[dt], cap,
+                     q.data_ptr(), k_blk.data_ptr(), v_blk.data_ptr(),
+                     k_cache.data_ptr(), v_cache.data_ptr(), cache_len.data_ptr(),
+                     float(scale) if scale else 0.0)
+
+
+def block_attend(view: int, q, k_blk, v_blk, k_cache, v_cache, cache_len,
+                 scale: Optional[float] = None, return_weights: bool = False):
+    """Dual-view block attention (Eq. 4 for VIEW_DIFFUSION; the causal verify pass
+    of Section 3.3 for VIEW_AR).  Returns out [B][K][Hq][d] float64, and with
+    `return_weights` also the softmax weights [B][K][Hq][max P_b + K]."""
+    a = _desc(q, k_blk, v_blk, k_cache, v_cache, cache_len, scale)
+    B, K, Hq, d = q.shape
+    out = torch.empty((B, K, Hq, d), dtype=torch.float64)
+    w = None
+    stride = 0
+    if return_weights:
+        stride = int(cache_len.max()) + K if B else K
+        w = torch.zeros((B, K, Hq, stride), dtype=torch.float64)
+    rc = lib().oracle_block_attend(ctypes.byref(a), view, out.data_ptr(),
+                                   w.data_ptr() if w is not None else None, stride)
+    if rc != 0:
+        raise RuntimeError(f"oracle_block_attend failed ({rc})")
+    return (out, w) if return_weights else out
+
+
+def block_attend_rows(view: int, rows: torch.Tensor, q, k_blk, v_blk, k_cache, v_cache,
+                      cache_len, scale: Optional[float] = None) -> torch.Tensor:
+    """Same attention for sampled rows only; rows int32 [n][3] = (b, i, hq).
+    Returns [n][d] float64."""
+    a = _desc(q, k_blk, v_blk, k_cache, v_cache, cache_len, scale)
+    rows = _check(rows.to(torch.int32).contiguous(), "rows")
+    out = torch.empty((rows.shape[0], q.shape[3]), dtype=torch.float64)
+    rc = lib().oracle_block_attend_rows(ctypes.byref(a), view, rows.data_ptr(),
+                                        rows.shape[0], out.data_ptr())
+    if rc != 0:
+        raise RuntimeError(f"oracle_block_attend_rows failed ({rc})")
+    return out
+
+
+def consensus_accept(logits: torch.Tensor, draft: torch.Tensor
+                     ) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor, torch.Tensor]:
+    """Greedy consensus (Eq. 8).  Returns (n_commit [B], committed [B][K],
+    ar_argmax [B][K], next_anchor [B]), all int32."""
+    _check(logits, "logits")
+    _check(draft, "draft")
+    B, K, V = logits.shape
+    if draft.dtype != torch.int32 or tuple(draft.shape) != (B, K):
+        raise ValueError("draft must be int32 [B][K]")
+    n = torch.empty(B, dtype=torch.int32)
+    com = torch.empty((B, K), dtype=torch.int32)
+    arg = torch.empty((B, K), dtype=torch.int32)
+    nxt = torch.empty(B, dtype=torch.int32)
+    rc = lib().oracle_consensus_accept(logits.data_ptr(), _DTYPE_CODE[logits.dtype],
+                                       draft.data_ptr(), B, K, V, n.data_ptr(),
+                                       com.data_ptr(), arg.data_ptr(), nxt.data_ptr())
+    if rc != 0:
+        raise RuntimeError(f"oracle_consensus_accept failed ({rc})")
+    return n, com, arg, nxt
+
+
+def kv_append(k_cache, v_cache, cache_len, k_blk, v_blk, n_commit, update_len: bool = True) -> int:
+    """KV commit, in place on k_cache / v_cache / cache_len.  Returns the C status
+    (0, or -3 if some sequence would overflow its capacity and was skipped)."""
+    for n_, t in (("k_cache", k_cache), ("v_cache", v_cache), ("cache_len", cache_len),
+                  ("k_blk", k_blk), ("v_blk", v_blk), ("n_commit", n_commit)):
+        _check(t, n_)
+    B, Hkv, cap, d = k_cache.shape
+    K = k_blk.shape[1]
+    return int(lib().oracle_kv_append(B, K, Hkv, d, cap, _DTYPE_CODE[k_cache.dtype],
+                                      k_cache.data_ptr(), v_cache.data_ptr(),
+                                      cache_len.data_ptr(), k_blk.data_ptr(),
+                                      v_blk.data_ptr(), n_commit.data_ptr(),
+                                      1 if update_len else 0))

@@ -1,0 +1,280 @@
+/*
+ * CPU oracle for the Orthrus generation-step hot path.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, fp64 statement of
+ * what the path computes, written from the paper.  It shares no code with the
+ * CUDA library and must never be called from the product path; only the test
+ * suite, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * Every function takes HOST pointers.  Tensors may be given as bf16 (raw
+ * 16-bit patterns), fp32 or fp64; each element is widened exactly to double
+ * before any arithmetic, and all sums are carried in double.
+ *
+ * Layouts (row-major):
+ *   q, out        [B][K][Hq][d]
+ *   k_blk, v_blk  [B][K][Hkv][d]
+ *   k_cache, v_cache [B][Hkv][capacity][d]
+ *   cache_len     [B] int32   (P_b = number of valid prefix positions)
+ *   logits        [B][K][V];  draft, committed, ar_argmax [B][K] int32
+ *
+ * Parity status: every function here is pinned by tests/test_oracle_pins.py
+ * (brute-force mask-matrix softmax, closed forms, K=1 reduction, permutation
+ * invariances, sequential greedy decoding of a toy model, byte-level append
+ * checks).  Nothing is "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORACLE_BF16 = 0, ORACLE_FP32 = 1, ORACLE_FP64 = 2 };
+enum { ORACLE_VIEW_DIFFUSION = 0, ORACLE_VIEW_AR = 1 };
+
+typedef struct {
+    int32_t batch, block, n_q_heads, n_kv_heads, head_dim;
+    int32_t dtype;          /* element type of q, k_blk, v_blk, k_cache, v_cache */
+    int64_t capacity;
+    const void *q, *k_blk, *v_blk, *k_cache, *v_cache;
+    const int32_t *cache_len;
+    double scale;           /* <= 0 selects 1/sqrt(head_dim), the scale of Eq. 4 */
+} oracle_attn_t;
+
+static double load_elem(const void *p, int dtype, int64_t idx)
+{
+    if (dtype == ORACLE_BF16) {
+        uint32_t bits = ((uint32_t)((const uint16_t *)p)[idx]) << 16;
+        float f;
+        memcpy(&f, &bits, sizeof f);
+        return (double)f;
+    }
+    if (dtype == ORACLE_FP32)
+        return (double)((const float *)p)[idx];
+    return ((const double *)p)[idx];
+}
+
+static size_t elem_size(int dtype)
+{
+    return dtype == ORACLE_BF16 ? 2 : dtype == ORACLE_FP32 ? 4 : 8;
+}
+
+/*
+ * One query row of the dual-view attention.
+ *
+ * Diffusion view (Eq. 4): the query of block position i, head hq, takes a softmax
+ * over the concatenation [K_AR || K_diff] = all P_b prefix rows of the shared
+ * cache followed by all K rows of the diffusion block (bidirectional inside the
+ * block, Section 3.2 rule (ii)), scaled by 1/sqrt(d_head), and averages
+ * [V_AR || V_diff] with those weights.
+ *
+ * AR view (Section 3.3, "Intra-Model Distribution Matching"): the block is fed
+ * through the ordinary causal model, so query i sees the whole prefix and block
+ * rows 0..i only.
+ *
+ * Grouped-query mapping: query head hq reads KV head hq / (Hq / Hkv).
+ *
+ * out_row: d doubles.  w_row: optional, P_b + K doubles (weights of masked block
+ * keys are written as exact zeros).  Returns 0, or -1 on allocation failure.
+ */
+static int attend_row(const oracle_attn_t *a, int view, int b, int hq, int i,
+                      double *out_row, double *w_row)
+{
+    const int d = a->head_dim, K = a->block, Hq = a->n_q_heads, Hkv = a->n_kv_heads;
+    const int G = Hq / Hkv;
+    const int h = hq / G;
+    const int64_t P = a->cache_len[b];
+    const int n_blk = (view == ORACLE_VIEW_DIFFUSION) ? K : i + 1;
+    const int64_t n = P + n_blk;
+    const double scale = a->scale > 0.0 ? a->scale : 1.0 / sqrt((double)d);
+
+    double *s = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    double *qv = (double *)malloc(sizeof(double) * (size_t)d);
+    if (!s || !qv) { free(s); free(qv); return -1; }
+
+    const int64_t q_off = (((int64_t)b * K + i) * Hq + hq) * d;
+    for (int c = 0; c < d; ++c) qv[c] = load_elem(a->q, a->dtype, q_off + c);
+
+    /* scores against the prefix cache rows */
+    const int64_t cache_base = ((int64_t)b * Hkv + h) * a->capacity * d;
+    for (int64_t j = 0; j < P; ++j) {
+        double acc = 0.0;
+        for (int c = 0; c < d; ++c)
+            acc += qv[c] * load_elem(a->k_cache, a->dtype, cache_base + j * d + c);
+        s[j] = acc * scale;
+    }
+    /* scores against the visible block rows */
+    for (int ip = 0; ip < n_blk; ++ip) {
+        const int64_t off = (((int64_t)b * K + ip) * Hkv + h) * d;
+        double acc = 0.0;
+        for (int c = 0; c < d; ++c)
+            acc += qv[c] * load_elem(a->k_blk, a->dtype, off + c);
+        s[P + ip] = acc * scale;
+    }
+
+    /* softmax */
+    double mx = -INFINITY;
+    for (int64_t j = 0; j < n; ++j) if (s[j] > mx) mx = s[j];
+    double den = 0.0;
+    for (int64_t j = 0; j < n; ++j) { s[j] = exp(s[j] - mx); den += s[j]; }
+    for (int64_t j = 0; j < n; ++j) s[j] /= den;
+
+    /* weighted average of the value rows */
+    for (int c = 0; c < d; ++c) out_row[c] = 0.0;
+    for (int64_t j = 0; j < P; ++j)
+        for (int c = 0; c < d; ++c)
+            out_row[c] += s[j] * load_elem(a->v_cache, a->dtype, cache_base + j * d + c);
+    for (int ip = 0; ip < n_blk; ++ip) {
+        const int64_t off = (((int64_t)b * K + ip) * Hkv + h) * d;
+        for (int c = 0; c < d; ++c)
+            out_row[c] += s[P + ip] * load_elem(a->v_blk, a->dtype, off + c);
+    }
+
+    if (w_row) {
+        for (int64_t j = 0; j < n; ++j) w_row[j] = s[j];
+        for (int64_t j = n; j < P + K; ++j) w_row[j] = 0.0;
+    }
+    free(s);
+    free(qv);
+    return 0;
+}
+
+/*
+ * Whole-tensor dual-view attention: out [B][K][Hq][d] doubles.
+ * weights (optional): [B][K][Hq][w_stride] doubles with w_stride >= max_b P_b + K;
+ * row (b,i,hq) holds its P_b + K weights followed by untouched slack.
+ */
+int oracle_block_attend(const oracle_attn_t *a, int view, double *out,
+                        double *weights, int64_t w_stride)
+{
+    const int B = a->batch, K = a->block, Hq = a->n_q_heads, d = a->head_dim;
+    if (a->n_kv_heads <= 0 || Hq % a->n_kv_heads != 0) return -2;
+    int rc = 0;
+    const int64_t rows = (int64_t)B * K * Hq;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < rows; ++r) {
+        const int hq = (int)(r % Hq);
+        const int i = (int)((r / Hq) % K);
+        const int b = (int)(r / ((int64_t)Hq * K));
+        double *w = weights ? weights + r * w_stride : NULL;
+        if (attend_row(a, view, b, hq, i, out + r * d, w) != 0) {
+#pragma omp atomic write
+            rc = -1;
+        }
+    }
+    return rc;
+}
+
+/*
+ * Sampled rows of the same attention, for sizes at which the whole tensor would
+ * take too long: rows[3*s + {0,1,2}] = (b, i, hq); out [n_rows][d] doubles.
+ */
+int oracle_block_attend_rows(const oracle_attn_t *a, int view, const int32_t *rows,
+                             int64_t n_rows, double *out)
+{
+    const int d = a->head_dim;
+    if (a->n_kv_heads <= 0 || a->n_q_heads % a->n_kv_heads != 0) return -2;
+    int rc = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t s = 0; s < n_rows; ++s) {
+        if (attend_row(a, view, rows[3 * s], rows[3 * s + 2], rows[3 * s + 1],
+                       out + s * d, NULL) != 0) {
+#pragma omp atomic write
+            rc = -1;
+        }
+    }
+    return rc;
+}
+
+/*
+ * Greedy consensus (Eq. 8 and the halt/commit rule of Section 3.3).
+ *
+ * Row i of the AR logits is conditioned on the anchor and drafts 0..i-1; its
+ * greedy token is g_i = argmax_v logits[b][i][v] (softmax is monotone, so the
+ * argmax of p_AR is the argmax of the logits; the smallest id wins ties; a NaN
+ * never wins).  Draft i is retained iff draft[i] == g_i.  Verification stops at
+ * the first mismatch; with m retained drafts the cycle commits those m tokens
+ * plus, when m < K, the correction token g_m.  When all K drafts agree there is
+ * no further verified row, so K tokens are committed.  Hence
+ *     n = min(m + 1, K),  committed = g_0..g_{n-1},  next anchor = g_{n-1},
+ * and 1 <= n <= K (at least one token per cycle, Section 4.2).
+ *
+ * Outputs: n_commit [B], committed [B][K] (-1 beyond n), ar_argmax [B][K],
+ * next_anchor [B].
+ */
+int oracle_consensus_accept(const void *logits, int dtype, const int32_t *draft,
+                            int32_t B, int32_t K, int32_t V,
+                            int32_t *n_commit, int32_t *committed,
+                            int32_t *ar_argmax, int32_t *next_anchor)
+{
+    if (B < 0 || K <= 0 || V <= 0) return -2;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < (int64_t)B * K; ++r) {
+        double best = -INFINITY;
+        int32_t arg = 0;
+        for (int32_t v = 0; v < V; ++v) {
+            const double x = load_elem(logits, dtype, r * V + v);
+            if (x > best) { best = x; arg = v; }
+        }
+        ar_argmax[r] = arg;
+    }
+    for (int32_t b = 0; b < B; ++b) {
+        const int32_t *g = ar_argmax + (int64_t)b * K;
+        const int32_t *y = draft + (int64_t)b * K;
+        int32_t m = 0;
+        while (m < K && y[m] == g[m]) ++m;
+        const int32_t n = (m + 1 < K) ? m + 1 : K;
+        n_commit[b] = n;
+        for (int32_t i = 0; i < K; ++i)
+            committed[(int64_t)b * K + i] = (i < n) ? g[i] : -1;
+        next_anchor[b] = g[n - 1];
+    }
+    return 0;
+}
+
+/*
+ * KV commit (Figure 2(b) and the last paragraph of Section 3.3): the AR-view
+ * K/V rows of the first n_b block positions join the shared cache right after
+ * the current prefix, for every KV head; the prefix grows by n_b.  Everything
+ * else in the cache is left byte-for-byte as it was.  The diffusion view's
+ * block KV is never stored.  Caches and block tensors are raw bytes of the
+ * given element type.  Returns -3 if a sequence would exceed its capacity
+ * (nothing is written for that sequence).
+ */
+int oracle_kv_append(int32_t B, int32_t K, int32_t Hkv, int32_t d, int64_t capacity,
+                     int dtype, void *k_cache, void *v_cache, int32_t *cache_len,
+                     const void *k_blk, const void *v_blk, const int32_t *n_commit,
+                     int update_len)
+{
+    const size_t es = elem_size(dtype);
+    const size_t row = (size_t)d * es;
+    int rc = 0;
+    for (int32_t b = 0; b < B; ++b) {
+        const int64_t P = cache_len[b];
+        const int32_t n = n_commit[b];
+        if (n < 0 || n > K || P < 0 || P + n > capacity) { rc = -3; continue; }
+        for (int32_t i = 0; i < n; ++i)
+            for (int32_t h = 0; h < Hkv; ++h) {
+                const size_t src = ((((size_t)b * K + i) * Hkv) + h) * row;
+                const size_t dst = ((((size_t)b * Hkv + h) * (size_t)capacity) + (size_t)(P + i)) * row;
+                memcpy((char *)k_cache + dst, (const char *)k_blk + src, row);
+                memcpy((char *)v_cache + dst, (const char *)v_blk + src, row);
+            }
+        if (update_len) cache_len[b] = (int32_t)(P + n);
+    }
+    return rc;
+}
+
+int oracle_num_threads(void)
+{
+    int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+    {
+#pragma omp master
+        n = omp_get_num_threads();
+    }
+#endif
+    return n;
+}
