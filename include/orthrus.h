@@ -1,0 +1,177 @@
+/*
+ * orthrus.h — C ABI of the B200 (sm_100a) hot path of the Orthrus generation step.
+ *
+ * One generation cycle (Section 3.3 of the paper) is, per transformer layer,
+ *   1. the diffusion view attending from a block of K positions to the shared
+ *      prefix KV cache and, bidirectionally, to the block itself   (Eq. 4),
+ *   2. the AR view verifying the same block causally over the same cache,
+ * then once per cycle
+ *   3. the greedy consensus between drafts and AR logits            (Eq. 8),
+ *   4. the commit of the accepted AR-view KV rows to the cache (Figure 2(b)).
+ * This library implements exactly those four operations as CUDA kernels.
+ *
+ * Conventions shared by every call
+ *   - Every data pointer is a DEVICE pointer owned by the caller, 16-byte
+ *     aligned, valid until the stream has passed the call.  Descriptors
+ *     (orthrus_layer_t) are HOST structs read during the call only.
+ *   - `stream` is a cudaStream_t passed as an opaque pointer (NULL = legacy
+ *     default stream).  Calls only enqueue work: they never synchronise, never
+ *     allocate, and keep no device state between calls.
+ *   - Problems the host can see (null or misaligned pointers, unsupported
+ *     shapes, a workspace that is too small) return an error code before
+ *     anything is launched.  Problems only the device can see (a cache_len
+ *     outside [0, capacity - K], an append past the capacity, a hardware wait
+ *     that ran out) never trap: the offending sequence is clamped or skipped
+ *     and a code is OR-ed into the status word at the start of the workspace,
+ *     which orthrus_read_status() fetches.
+ *   - Tensors are row-major, innermost dimension last:
+ *       q_*, out           [B][K][Hq][d]
+ *       k_*_blk, v_*_blk   [B][K][Hkv][d]
+ *       k_cache, v_cache   [B][Hkv][capacity][d]
+ *       ar_logits          [B][K][V]
+ *       draft, committed, ar_argmax  [B][K] int32;  n_commit, next_anchor, cache_len [B] int32
+ *     Query head hq reads KV head hq / (Hq / Hkv).
+ *   - dtype ORTHRUS_BF16: bf16 inputs/outputs, fp32 softmax and accumulation.
+ *     dtype ORTHRUS_FP32: fp32 everywhere (a slow test mode).
+ */
+#ifndef ORTHRUS_H_
+#define ORTHRUS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ORTHRUS_OK = 0,
+    ORTHRUS_ERR_INVALID_ARG = 1,  /* null/misaligned pointer, bad size            */
+    ORTHRUS_ERR_UNSUPPORTED = 2,  /* shape or dtype outside the supported set     */
+    ORTHRUS_ERR_CAPACITY = 3,     /* max_len_hint + block exceeds capacity        */
+    ORTHRUS_ERR_WORKSPACE = 4,    /* workspace smaller than *_workspace_bytes()   */
+    ORTHRUS_ERR_CUDA = 5          /* a CUDA runtime call failed                   */
+} orthrus_status_t;
+
+/* bits of the device status word (first int32 of the workspace) */
+enum {
+    ORTHRUS_DEV_BAD_CACHE_LEN = 1,   /* cache_len[b] outside [0, capacity-K]: clamped      */
+    ORTHRUS_DEV_APPEND_OVERFLOW = 2, /* cache_len[b]+n_commit[b] > capacity, or n_commit[b]
+                                        outside [0,K]: that sequence was not appended       */
+    ORTHRUS_DEV_WAIT_TIMEOUT = 4     /* a bounded hardware wait expired; outputs undefined  */
+};
+
+typedef enum { ORTHRUS_BF16 = 0, ORTHRUS_FP32 = 1 } orthrus_dtype_t;
+
+/* One layer's shared KV cache plus the shape of the block attending to it. */
+typedef struct {
+    int32_t batch;          /* B >= 1                                               */
+    int32_t n_q_heads;      /* Hq, a multiple of n_kv_heads                         */
+    int32_t n_kv_heads;     /* Hkv                                                  */
+    int32_t head_dim;       /* d in {32, 64, 128, 256}; tensor-core paths: 64, 128  */
+    int32_t block;          /* K, 1..64                                             */
+    int32_t dtype;          /* orthrus_dtype_t of q, out, block KV and cache        */
+    int64_t capacity;       /* positions per (sequence, KV head) in the cache       */
+    void *k_cache;          /* device [B][Hkv][capacity][d]                         */
+    void *v_cache;          /* device [B][Hkv][capacity][d]                         */
+    int32_t *cache_len;     /* device [B]: prefix length P_b, 0 <= P_b <= cap - K   */
+    int32_t max_len_hint;   /* host upper bound on every P_b; sizes the split-KV
+                               grid.  0 means capacity - block                      */
+    float softmax_scale;    /* 0 selects 1/sqrt(head_dim), the scale of Eq. 4       */
+} orthrus_layer_t;
+
+/*
+ * Bytes of workspace the two attention calls (and orthrus_kv_append) need for
+ * this layer shape: a 256-byte header holding the status word, followed by the
+ * split-KV partial results.  Returns 0 for an invalid descriptor.
+ */
+size_t orthrus_attend_workspace_bytes(const orthrus_layer_t *layer);
+
+/*
+ * Zeroes the workspace header (status word).  Call once after allocating a
+ * workspace and whenever the status word should be cleared.
+ */
+orthrus_status_t orthrus_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Diffusion-view block attention, Eq. 4: for every sequence b, query head hq and
+ * block position i,
+ *   out[b][i][hq] = softmax_j( q_diff[b][i][hq] . key_j * scale ) applied to value_j,
+ * where j runs over the P_b cache rows of KV head hq/(Hq/Hkv) followed by ALL K
+ * rows of the diffusion block (k_diff_blk, v_diff_blk): the block is
+ * bidirectional (Section 3.2, viewing rule (ii)).  The block KV is transient: it
+ * is read here and never stored.
+ */
+orthrus_status_t orthrus_diffusion_block_attend(const orthrus_layer_t *layer,
+        const void *q_diff, const void *k_diff_blk, const void *v_diff_blk, void *out,
+        void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * AR-view verify attention (Section 3.3, "Intra-Model Distribution Matching"):
+ * the same as above with the AR-view block tensors, except that the block is
+ * causal: position i sees the P_b cache rows and block rows 0..i only, which is
+ * what the frozen causal model computes for the materialised block.
+ */
+orthrus_status_t orthrus_ar_verify_attend(const orthrus_layer_t *layer,
+        const void *q_ar, const void *k_ar_blk, const void *v_ar_blk, void *out,
+        void *workspace, size_t workspace_bytes, void *stream);
+
+/* Workspace bytes for orthrus_consensus_accept (header + per-row partial maxima). */
+size_t orthrus_consensus_workspace_bytes(int32_t batch, int32_t block, int32_t vocab);
+
+/*
+ * Greedy consensus, Eq. 8 with the halt/commit rule of Section 3.3.
+ *   ar_argmax[b][i] = smallest v maximising ar_logits[b][i][v]   (NaN never wins)
+ *   m_b       = number of leading positions with draft[b][i] == ar_argmax[b][i]
+ *   n_commit[b] = min(m_b + 1, K)   (agreeing drafts plus the correction token;
+ *                                    K when the whole block agrees; always >= 1)
+ *   committed[b][i] = ar_argmax[b][i] for i < n_commit[b], else -1
+ *   next_anchor[b]  = ar_argmax[b][n_commit[b] - 1]
+ * `dtype` is the element type of ar_logits.  All outputs are bit-exact.
+ */
+orthrus_status_t orthrus_consensus_accept(const void *ar_logits, int32_t dtype,
+        const int32_t *draft, int32_t batch, int32_t block, int32_t vocab,
+        int32_t *n_commit, int32_t *committed, int32_t *ar_argmax, int32_t *next_anchor,
+        void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * KV commit (Figure 2(b); last paragraph of Section 3.3): for every sequence b,
+ * KV head h and i < n_commit[b],
+ *   k_cache[b][h][P_b + i] = k_ar_blk[b][i][h]   (likewise v),
+ * a byte copy; with update_len != 0, cache_len[b] += n_commit[b] afterwards.
+ * update_len = 0 lets several layers that share one cache_len array be appended
+ * before the length is bumped by the last of them.  Rows outside
+ * [P_b, P_b + n_commit[b]) are not touched.  `workspace` may be NULL; if given,
+ * overflow is reported through its status word.
+ */
+orthrus_status_t orthrus_kv_append(const orthrus_layer_t *layer, const void *k_ar_blk,
+        const void *v_ar_blk, const int32_t *n_commit, int32_t update_len,
+        void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Copies the device status word to *host_status and waits for the stream (the
+ * only call here that synchronises).  0 means no device-side problem so far.
+ */
+orthrus_status_t orthrus_read_status(const void *workspace, void *stream, int32_t *host_status);
+
+/*
+ * Kernel-path selection for measurements: "auto" (default), "simt", "mma" or
+ * "tcgen05".  A path that does not support the shape falls back to the next
+ * more general one.  Returns ORTHRUS_ERR_INVALID_ARG for an unknown name.
+ * Also settable through the environment variable ORTHRUS_FORCE_PATH.
+ */
+orthrus_status_t orthrus_set_path(const char *name);
+
+/* Name of the kernel path the last attention call on this thread took. */
+const char *orthrus_last_path(void);
+
+/* Number of kernels launched by this library in this process so far. */
+int64_t orthrus_launch_count(void);
+
+const char *orthrus_status_string(orthrus_status_t status);
+int32_t orthrus_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ORTHRUS_H_ */

@@ -1,0 +1,193 @@
+"""Thin ctypes binding of liborthrus.so (argument marshalling only).
+
+Every function has the name of the C entry point it calls; tensors are torch CUDA
+tensors whose device pointers are handed over unchanged.  torch is used for device
+memory and streams, nothing else.  There is no fallback: if the library has not
+been built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liborthrus.so")
+
+OK = 0
+BF16, FP32 = 0, 1
+DEV_BAD_CACHE_LEN, DEV_APPEND_OVERFLOW, DEV_WAIT_TIMEOUT = 1, 2, 4
+
+EXPORTS = [
+    "orthrus_attend_workspace_bytes", "orthrus_workspace_init",
+    "orthrus_diffusion_block_attend", "orthrus_ar_verify_attend",
+    "orthrus_consensus_workspace_bytes", "orthrus_consensus_accept",
+    "orthrus_kv_append", "orthrus_read_status", "orthrus_set_path", "orthrus_last_path",
+    "orthrus_launch_count", "orthrus_status_string", "orthrus_version",
+]
+
+
+class OrthrusError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = _lib.orthrus_status_string(code).decode() if _lib is not None else str(code)
+        super().__init__(f"{where}: {msg} (status {code})")
+
+
+class Layer(ctypes.Structure):
+    """Mirror of orthrus_layer_t."""
+    _fields_ = [("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
+                ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("block", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("capacity", ctypes.c_int64), ("k_cache", ctypes.c_void_p),
+                ("v_cache", ctypes.c_void_p), ("cache_len", ctypes.c_void_p),
+                ("max_len_hint", ctypes.c_int32), ("softmax_scale", ctypes.c_float)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2605_12825_b200.build` "
+            "(there is no CPU or PyTorch fallback for the Orthrus kernels)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    LP = ctypes.POINTER(Layer)
+    lib.orthrus_attend_workspace_bytes.restype = sz
+    lib.orthrus_attend_workspace_bytes.argtypes = [LP]
+    lib.orthrus_workspace_init.restype = ctypes.c_int
+    lib.orthrus_workspace_init.argtypes = [vp, sz, vp]
+    for name in ("orthrus_diffusion_block_attend", "orthrus_ar_verify_attend"):
+        f = getattr(lib, name)
+        f.restype = ctypes.c_int
+        f.argtypes = [LP, vp, vp, vp, vp, vp, sz, vp]
+    lib.orthrus_consensus_workspace_bytes.restype = sz
+    lib.orthrus_consensus_workspace_bytes.argtypes = [i32, i32, i32]
+    lib.orthrus_consensus_accept.restype = ctypes.c_int
+    lib.orthrus_consensus_accept.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+    lib.orthrus_kv_append.restype = ctypes.c_int
+    lib.orthrus_kv_append.argtypes = [LP, vp, vp, vp, i32, vp, sz, vp]
+    lib.orthrus_read_status.restype = ctypes.c_int
+    lib.orthrus_read_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
+    lib.orthrus_set_path.restype = ctypes.c_int
+    lib.orthrus_set_path.argtypes = [ctypes.c_char_p]
+    lib.orthrus_last_path.restype = ctypes.c_char_p
+    lib.orthrus_launch_count.restype = i64
+    lib.orthrus_status_string.restype = ctypes.c_char_p
+    lib.orthrus_status_string.argtypes = [ctypes.c_int]
+    lib.orthrus_version.restype = i32
+    return lib
+
+
+_lib = None
+_lib = _load()
+
+
+def lib() -> ctypes.CDLL:
+    return _lib
+
+
+def dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.bfloat16:
+        return BF16
+    if dt == torch.float32:
+        return FP32
+    raise TypeError(f"unsupported dtype {dt}")
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise OrthrusError(code, where)
+
+
+def make_layer(k_cache: torch.Tensor, v_cache: torch.Tensor, cache_len: torch.Tensor,
+               n_q_heads: int, block: int, max_len_hint: int = 0,
+               softmax_scale: float = 0.0) -> Layer:
+    """Describe one layer's shared cache ([B][Hkv][capacity][d]) and block shape."""
+    B, Hkv, cap, d = k_cache.shape
+    return Layer(B, n_q_heads, Hkv, d, block, dtype_code(k_cache.dtype), cap,
+                 k_cache.data_ptr(), v_cache.data_ptr(), cache_len.data_ptr(),
+                 max_len_hint, softmax_scale)
+
+
+def orthrus_attend_workspace_bytes(layer: Layer) -> int:
+    return int(_lib.orthrus_attend_workspace_bytes(ctypes.byref(layer)))
+
+
+def orthrus_workspace_init(workspace: torch.Tensor, stream=None) -> None:
+    _check(_lib.orthrus_workspace_init(workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                       _stream(stream)), "orthrus_workspace_init")
+
+
+def new_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    orthrus_workspace_init(ws)
+    return ws
+
+
+def orthrus_diffusion_block_attend(layer: Layer, q_diff, k_diff_blk, v_diff_blk, out, workspace,
+                                   stream=None) -> None:
+    _check(_lib.orthrus_diffusion_block_attend(
+        ctypes.byref(layer), _ptr(q_diff), _ptr(k_diff_blk), _ptr(v_diff_blk), _ptr(out),
+        _ptr(workspace), workspace.numel(), _stream(stream)), "orthrus_diffusion_block_attend")
+
+
+def orthrus_ar_verify_attend(layer: Layer, q_ar, k_ar_blk, v_ar_blk, out, workspace,
+                             stream=None) -> None:
+    _check(_lib.orthrus_ar_verify_attend(
+        ctypes.byref(layer), _ptr(q_ar), _ptr(k_ar_blk), _ptr(v_ar_blk), _ptr(out),
+        _ptr(workspace), workspace.numel(), _stream(stream)), "orthrus_ar_verify_attend")
+
+
+def orthrus_consensus_workspace_bytes(batch: int, block: int, vocab: int) -> int:
+    return int(_lib.orthrus_consensus_workspace_bytes(batch, block, vocab))
+
+
+def orthrus_consensus_accept(ar_logits, draft, n_commit, committed, ar_argmax, next_anchor,
+                             workspace, stream=None) -> None:
+    B, K, V = ar_logits.shape
+    _check(_lib.orthrus_consensus_accept(
+        _ptr(ar_logits), dtype_code(ar_logits.dtype), _ptr(draft), B, K, V, _ptr(n_commit),
+        _ptr(committed), _ptr(ar_argmax), _ptr(next_anchor), _ptr(workspace), workspace.numel(),
+        _stream(stream)), "orthrus_consensus_accept")
+
+
+def orthrus_kv_append(layer: Layer, k_ar_blk, v_ar_blk, n_commit, update_len: bool = True,
+                      workspace=None, stream=None) -> None:
+    _check(_lib.orthrus_kv_append(
+        ctypes.byref(layer), _ptr(k_ar_blk), _ptr(v_ar_blk), _ptr(n_commit),
+        1 if update_len else 0, _ptr(workspace), 0 if workspace is None else workspace.numel(),
+        _stream(stream)), "orthrus_kv_append")
+
+
+def orthrus_read_status(workspace, stream=None) -> int:
+    out = ctypes.c_int32(-1)
+    _check(_lib.orthrus_read_status(workspace.data_ptr(), _stream(stream), ctypes.byref(out)),
+           "orthrus_read_status")
+    return int(out.value)
+
+
+def orthrus_set_path(name: str) -> None:
+    _check(_lib.orthrus_set_path(name.encode()), "orthrus_set_path")
+
+
+def orthrus_last_path() -> str:
+    return _lib.orthrus_last_path().decode()
+
+
+def orthrus_launch_count() -> int:
+    return int(_lib.orthrus_launch_count())
+
+
+def orthrus_version() -> int:
+    return int(_lib.orthrus_version())

@@ -1,0 +1,278 @@
+// C-ABI entry points: argument validation, split-KV planning, kernel-path dispatch.
+#include <atomic>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include "common.cuh"
+
+namespace orthrus {
+
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+enum Path { PATH_AUTO = 0, PATH_SIMT, PATH_MMA, PATH_TCGEN05 };
+static std::atomic<int> g_path{-1};
+static thread_local const char *t_last_path = "none";
+
+static int parse_path(const char *s)
+{
+    if (!s || !*s || !strcmp(s, "auto")) return PATH_AUTO;
+    if (!strcmp(s, "simt")) return PATH_SIMT;
+    if (!strcmp(s, "mma")) return PATH_MMA;
+    if (!strcmp(s, "tcgen05")) return PATH_TCGEN05;
+    return -1;
+}
+
+static int current_path()
+{
+    int v = g_path.load();
+    if (v < 0) {
+        v = parse_path(getenv("ORTHRUS_FORCE_PATH"));
+        if (v < 0) v = PATH_AUTO;
+        g_path.store(v);
+    }
+    return v;
+}
+
+static int env_int(const char *name, int dflt)
+{
+    const char *s = getenv(name);
+    if (!s || !*s) return dflt;
+    const int v = atoi(s);
+    return v > 0 ? v : dflt;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+static orthrus_status_t check_layer(const orthrus_layer_t *L)
+{
+    if (!L) return ORTHRUS_ERR_INVALID_ARG;
+    if (L->batch < 1 || L->n_q_heads < 1 || L->n_kv_heads < 1 || L->block < 1 || L->capacity < 1)
+        return ORTHRUS_ERR_INVALID_ARG;
+    if (L->n_q_heads % L->n_kv_heads != 0) return ORTHRUS_ERR_INVALID_ARG;
+    if (L->dtype != ORTHRUS_BF16 && L->dtype != ORTHRUS_FP32) return ORTHRUS_ERR_UNSUPPORTED;
+    if (L->head_dim != 32 && L->head_dim != 64 && L->head_dim != 128 && L->head_dim != 256)
+        return ORTHRUS_ERR_UNSUPPORTED;
+    if (L->block > 64) return ORTHRUS_ERR_UNSUPPORTED;
+    if (L->max_len_hint < 0 || !(L->softmax_scale >= 0.f) || std::isinf(L->softmax_scale))
+        return ORTHRUS_ERR_INVALID_ARG;
+    if (L->block > L->capacity) return ORTHRUS_ERR_CAPACITY;
+    if (L->capacity > 0x7fffffffLL) return ORTHRUS_ERR_UNSUPPORTED;
+    if ((long long)L->max_len_hint + L->block > L->capacity) return ORTHRUS_ERR_CAPACITY;
+    return ORTHRUS_OK;
+}
+
+static int max_len_of(const orthrus_layer_t *L)
+{
+    return L->max_len_hint > 0 ? L->max_len_hint : (int)(L->capacity - L->block);
+}
+
+// Split-KV plan: a pure function of the descriptor (and of two tuning variables read
+// from the environment), so that the workspace query and the launch always agree.
+struct Plan { int chunk, n_splits; };
+
+static Plan make_plan(const orthrus_layer_t *L)
+{
+    const int tile = 64;
+    const int units = L->batch * L->n_kv_heads;
+    const int max_len = max_len_of(L);
+    const int tiles = max_len > 0 ? (max_len + tile - 1) / tile : 1;
+    const int target = env_int("ORTHRUS_TARGET_CTAS", 2 * kNumSMs);
+    const int min_chunk_tiles = env_int("ORTHRUS_MIN_CHUNK_TILES", 4);
+    int splits = (target + units - 1) / units;
+    const int forced = env_int("ORTHRUS_SPLITS", 0);
+    if (forced > 0) splits = forced;
+    int max_splits = tiles / min_chunk_tiles;
+    if (forced > 0) max_splits = tiles;
+    if (max_splits < 1) max_splits = 1;
+    if (max_splits > kMaxSplits) max_splits = kMaxSplits;
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    const int chunk_tiles = (tiles + splits - 1) / splits;
+    Plan pl;
+    pl.chunk = chunk_tiles * tile;
+    pl.n_splits = max_len > 0 ? (max_len + pl.chunk - 1) / pl.chunk : 1;
+    return pl;
+}
+
+static size_t partial_bytes(const orthrus_layer_t *L, const Plan &pl, size_t *ml_off)
+{
+    const size_t units = (size_t)L->batch * L->n_kv_heads;
+    const size_t M = (size_t)(L->n_q_heads / L->n_kv_heads) * L->block;
+    if (pl.n_splits == 1) { if (ml_off) *ml_off = 0; return 0; }
+    const size_t o_bytes = units * pl.n_splits * M * L->head_dim * sizeof(float);
+    const size_t ml_bytes = units * pl.n_splits * M * 2 * sizeof(float);
+    if (ml_off) *ml_off = o_bytes;
+    return o_bytes + ml_bytes;
+}
+
+static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void *q,
+                               const void *k_blk, const void *v_blk, void *out, void *ws,
+                               size_t ws_bytes, void *stream)
+{
+    orthrus_status_t st = check_layer(L);
+    if (st != ORTHRUS_OK) return st;
+    if (!q || !k_blk || !v_blk || !out || !ws || !L->k_cache || !L->v_cache || !L->cache_len)
+        return ORTHRUS_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out) ||
+        !aligned16(ws) || !aligned16(L->k_cache) || !aligned16(L->v_cache) ||
+        (reinterpret_cast<uintptr_t>(L->cache_len) & 3))
+        return ORTHRUS_ERR_INVALID_ARG;
+    const Plan pl = make_plan(L);
+    size_t ml_off = 0;
+    const size_t need = kHeaderBytes + partial_bytes(L, pl, &ml_off);
+    if (ws_bytes < need) return ORTHRUS_ERR_WORKSPACE;
+
+    AttnParams p;
+    p.q = q; p.k_blk = k_blk; p.v_blk = v_blk; p.k_cache = L->k_cache; p.v_cache = L->v_cache;
+    p.cache_len = L->cache_len; p.out = out;
+    unsigned char *base = static_cast<unsigned char *>(ws);
+    p.status = reinterpret_cast<int32_t *>(base);
+    p.part_o = reinterpret_cast<float *>(base + kHeaderBytes);
+    p.part_ml = reinterpret_cast<float *>(base + kHeaderBytes + ml_off);
+    p.B = L->batch; p.K = L->block; p.Hq = L->n_q_heads; p.Hkv = L->n_kv_heads;
+    p.G = p.Hq / p.Hkv; p.M = p.G * p.K; p.d = L->head_dim; p.capacity = L->capacity;
+    p.chunk = pl.chunk; p.n_splits = pl.n_splits; p.causal = causal;
+    const float scale = L->softmax_scale > 0.f ? L->softmax_scale : 1.f / sqrtf((float)p.d);
+    p.scale_log2 = scale * 1.4426950408889634f;
+
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const int want = current_path();
+    cudaError_t e;
+    if (want != PATH_SIMT && mma_path_supports(p, L->dtype)) {
+        t_last_path = "mma";
+        e = launch_attend_mma(p, cs);
+    } else {
+        t_last_path = "simt";
+        e = launch_attend_simt(p, L->dtype, cs);
+    }
+    if (e != cudaSuccess) return ORTHRUS_ERR_CUDA;
+    if (pl.n_splits > 1) {
+        e = launch_combine(p, L->dtype, cs);
+        if (e != cudaSuccess) return ORTHRUS_ERR_CUDA;
+    }
+    return ORTHRUS_OK;
+}
+
+}  // namespace orthrus
+
+using namespace orthrus;
+
+extern "C" {
+
+size_t orthrus_attend_workspace_bytes(const orthrus_layer_t *layer)
+{
+    if (check_layer(layer) != ORTHRUS_OK) return 0;
+    return kHeaderBytes + partial_bytes(layer, make_plan(layer), nullptr);
+}
+
+orthrus_status_t orthrus_workspace_init(void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!workspace || workspace_bytes < (size_t)kHeaderBytes) return ORTHRUS_ERR_INVALID_ARG;
+    return cudaMemsetAsync(workspace, 0, kHeaderBytes, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+}
+
+orthrus_status_t orthrus_diffusion_block_attend(const orthrus_layer_t *layer, const void *q_diff,
+        const void *k_diff_blk, const void *v_diff_blk, void *out, void *workspace,
+        size_t workspace_bytes, void *stream)
+{
+    return attend(layer, 0, q_diff, k_diff_blk, v_diff_blk, out, workspace, workspace_bytes, stream);
+}
+
+orthrus_status_t orthrus_ar_verify_attend(const orthrus_layer_t *layer, const void *q_ar,
+        const void *k_ar_blk, const void *v_ar_blk, void *out, void *workspace,
+        size_t workspace_bytes, void *stream)
+{
+    return attend(layer, 1, q_ar, k_ar_blk, v_ar_blk, out, workspace, workspace_bytes, stream);
+}
+
+size_t orthrus_consensus_workspace_bytes(int32_t batch, int32_t block, int32_t vocab)
+{
+    if (batch < 1 || block < 1 || vocab < 1) return 0;
+    return kHeaderBytes + (size_t)batch * block * consensus_segments(batch, block, vocab) * 8;
+}
+
+orthrus_status_t orthrus_consensus_accept(const void *ar_logits, int32_t dtype, const int32_t *draft,
+        int32_t batch, int32_t block, int32_t vocab, int32_t *n_commit, int32_t *committed,
+        int32_t *ar_argmax, int32_t *next_anchor, void *workspace, size_t workspace_bytes,
+        void *stream)
+{
+    if (batch < 1 || block < 1 || vocab < 1) return ORTHRUS_ERR_INVALID_ARG;
+    if (dtype != ORTHRUS_BF16 && dtype != ORTHRUS_FP32) return ORTHRUS_ERR_UNSUPPORTED;
+    if (block > 1024 || (long long)batch * block > 65535) return ORTHRUS_ERR_UNSUPPORTED;
+    if (!ar_logits || !draft || !n_commit || !committed || !ar_argmax || !next_anchor || !workspace)
+        return ORTHRUS_ERR_INVALID_ARG;
+    const size_t es = dtype == ORTHRUS_FP32 ? 4 : 2;
+    if ((reinterpret_cast<uintptr_t>(ar_logits) & (es - 1)) || !aligned16(workspace) ||
+        ((reinterpret_cast<uintptr_t>(draft) | reinterpret_cast<uintptr_t>(n_commit) |
+          reinterpret_cast<uintptr_t>(committed) | reinterpret_cast<uintptr_t>(ar_argmax) |
+          reinterpret_cast<uintptr_t>(next_anchor)) & 3))
+        return ORTHRUS_ERR_INVALID_ARG;
+    if (workspace_bytes < orthrus_consensus_workspace_bytes(batch, block, vocab))
+        return ORTHRUS_ERR_WORKSPACE;
+    const int n_seg = consensus_segments(batch, block, vocab);
+    cudaError_t e = launch_consensus(ar_logits, dtype, draft, batch, block, vocab, n_commit, committed,
+                                     ar_argmax, next_anchor,
+                                     static_cast<unsigned char *>(workspace) + kHeaderBytes, n_seg,
+                                     static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+}
+
+orthrus_status_t orthrus_kv_append(const orthrus_layer_t *layer, const void *k_ar_blk,
+        const void *v_ar_blk, const int32_t *n_commit, int32_t update_len, void *workspace,
+        size_t workspace_bytes, void *stream)
+{
+    orthrus_status_t st = check_layer(layer);
+    if (st != ORTHRUS_OK) return st;
+    if (!k_ar_blk || !v_ar_blk || !n_commit || !layer->k_cache || !layer->v_cache || !layer->cache_len)
+        return ORTHRUS_ERR_INVALID_ARG;
+    if (!aligned16(k_ar_blk) || !aligned16(v_ar_blk) || !aligned16(layer->k_cache) ||
+        !aligned16(layer->v_cache) || (reinterpret_cast<uintptr_t>(n_commit) & 3) ||
+        (reinterpret_cast<uintptr_t>(layer->cache_len) & 3))
+        return ORTHRUS_ERR_INVALID_ARG;
+    if (workspace && (workspace_bytes < (size_t)kHeaderBytes || !aligned16(workspace)))
+        return ORTHRUS_ERR_WORKSPACE;
+    cudaError_t e = launch_kv_append(*layer, k_ar_blk, v_ar_blk, n_commit, update_len,
+                                     static_cast<int32_t *>(workspace),
+                                     static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+}
+
+orthrus_status_t orthrus_read_status(const void *workspace, void *stream, int32_t *host_status)
+{
+    if (!workspace || !host_status) return ORTHRUS_ERR_INVALID_ARG;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(host_status, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+        return ORTHRUS_ERR_CUDA;
+    return cudaStreamSynchronize(cs) == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+}
+
+orthrus_status_t orthrus_set_path(const char *name)
+{
+    const int v = parse_path(name);
+    if (v < 0) return ORTHRUS_ERR_INVALID_ARG;
+    g_path.store(v);
+    return ORTHRUS_OK;
+}
+
+const char *orthrus_last_path(void) { return t_last_path; }
+
+int64_t orthrus_launch_count(void) { return g_launches.load(); }
+
+const char *orthrus_status_string(orthrus_status_t status)
+{
+    switch (status) {
+    case ORTHRUS_OK: return "ok";
+    case ORTHRUS_ERR_INVALID_ARG: return "invalid argument";
+    case ORTHRUS_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case ORTHRUS_ERR_CAPACITY: return "block does not fit in the cache capacity";
+    case ORTHRUS_ERR_WORKSPACE: return "workspace too small";
+    case ORTHRUS_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown status";
+}
+
+int32_t orthrus_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,69 @@
+// Shared declarations of the Orthrus CUDA library: kernel parameter blocks,
+// workspace layout and the launchers each translation unit exports.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "orthrus.h"
+
+namespace orthrus {
+
+constexpr int kHeaderBytes = 256;       // workspace header; int32 status word at offset 0
+constexpr int kMaxSplits = 64;
+constexpr int kNumSMs = 148;
+
+// Parameters common to every attention kernel.  Rows of one (sequence, KV head)
+// unit are ordered r = i * G + g  (block position i, head g within the group), so
+// that the G query heads sharing a KV head and all K block positions form one tile
+// of M = G * K rows.
+struct AttnParams {
+    const void *q, *k_blk, *v_blk, *k_cache, *v_cache;
+    const int32_t *cache_len;
+    void *out;
+    float *part_o;      // [unit][split][M][d]   unnormalised partial outputs
+    float *part_ml;     // [unit][split][M][2]   running max (log2 domain), running sum
+    int32_t *status;    // device status word
+    int B, K, Hq, Hkv, G, M, d;
+    long long capacity;
+    int chunk;          // prefix positions per split
+    int n_splits;       // grid extent along the split axis
+    int causal;         // 0: diffusion view (bidirectional block), 1: AR view (causal block)
+    float scale_log2;   // softmax scale times log2(e)
+};
+
+// split s of a unit covers prefix positions [s*chunk, min((s+1)*chunk, P)); the split
+// that holds the last prefix position (split 0 for an empty prefix) also takes the
+// block keys.  Splits beyond it do nothing.
+__host__ __device__ inline int last_split(int P, int chunk) {
+    return P <= 0 ? 0 : (P - 1) / chunk;
+}
+
+__device__ inline int clamp_cache_len(const AttnParams &p, int b) {
+    int P = p.cache_len[b];
+    long long hi = p.capacity - p.K;
+    if (P < 0 || P > hi) {
+        if (p.status) atomicOr(p.status, ORTHRUS_DEV_BAD_CACHE_LEN);
+        P = P < 0 ? 0 : (int)hi;
+    }
+    return P;
+}
+
+// launchers (each returns the cudaError of its launches)
+cudaError_t launch_attend_simt(const AttnParams &p, int dtype, cudaStream_t st);
+bool mma_path_supports(const AttnParams &p, int dtype);
+cudaError_t launch_attend_mma(const AttnParams &p, cudaStream_t st);
+int mma_tile_positions();
+cudaError_t launch_combine(const AttnParams &p, int dtype, cudaStream_t st);
+
+cudaError_t launch_consensus(const void *logits, int dtype, const int32_t *draft, int B, int K,
+                             int V, int32_t *n_commit, int32_t *committed, int32_t *ar_argmax,
+                             int32_t *next_anchor, void *partials, int n_seg, cudaStream_t st);
+int consensus_segments(int B, int K, int V);
+
+cudaError_t launch_kv_append(const orthrus_layer_t &L, const void *k_blk, const void *v_blk,
+                             const int32_t *n_commit, int update_len, int32_t *status,
+                             cudaStream_t st);
+
+void count_launch(int n = 1);
+
+}  // namespace orthrus

@@ -1,0 +1,88 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the header
+declares, and rejects host-detectable misuse before launching anything."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2605_12825_b200 import build
+    build.build()
+    from paper_2605_12825_b200 import binding
+    return binding
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "orthrus.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(orthrus_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_symbols()
+    assert "orthrus_diffusion_block_attend" in names and "orthrus_kv_append" in names
+    for n in names:
+        assert hasattr(lib.lib(), n), n
+    assert set(names) == set(lib.EXPORTS)
+    assert lib.orthrus_version() >= 100
+
+
+def test_status_strings(lib):
+    s = {lib.lib().orthrus_status_string(c).decode() for c in range(6)}
+    assert len(s) == 6
+
+
+def _layer(lib, **kw):
+    d = dict(batch=1, n_q_heads=8, n_kv_heads=2, head_dim=64, block=8, dtype=0, capacity=1024,
+             k_cache=0x1000, v_cache=0x2000, cache_len=0x3000, max_len_hint=512, softmax_scale=0.0)
+    d.update(kw)
+    return lib.Layer(*[d[f[0]] for f in lib.Layer._fields_])
+
+
+def test_workspace_query_and_plan(lib):
+    assert lib.orthrus_attend_workspace_bytes(_layer(lib)) >= 256
+    assert lib.orthrus_attend_workspace_bytes(_layer(lib, n_q_heads=7)) == 0      # Hq % Hkv
+    assert lib.orthrus_attend_workspace_bytes(_layer(lib, head_dim=48)) == 0
+    assert lib.orthrus_attend_workspace_bytes(_layer(lib, max_len_hint=1020)) == 0  # + K > cap
+    big = lib.orthrus_attend_workspace_bytes(
+        _layer(lib, n_q_heads=32, n_kv_heads=8, head_dim=128, block=16, capacity=4160,
+               max_len_hint=4096))
+    assert big > 256      # long prefix, few units: split-KV partials are needed
+    assert lib.orthrus_consensus_workspace_bytes(1, 16, 151936) > 256
+    assert lib.orthrus_consensus_workspace_bytes(0, 16, 10) == 0
+
+
+@pytest.mark.parametrize("bad,code", [
+    (dict(n_q_heads=7), 1), (dict(head_dim=48), 2), (dict(block=65), 2), (dict(dtype=5), 2),
+    (dict(max_len_hint=1020), 3), (dict(k_cache=0), 1), (dict(k_cache=0x1008), 1),
+    (dict(softmax_scale=-1.0), 1),
+])
+def test_attend_rejects_bad_descriptors_before_launch(lib, bad, code):
+    L = _layer(lib, **bad)
+    n0 = lib.orthrus_launch_count()
+    for fn in (lib.lib().orthrus_diffusion_block_attend, lib.lib().orthrus_ar_verify_attend):
+        rc = fn(ctypes.byref(L), 0x4000, 0x5000, 0x6000, 0x7000, 0x8000, 1 << 30, None)
+        assert rc == code
+    assert lib.orthrus_launch_count() == n0
+
+
+def test_null_and_small_workspace(lib):
+    L = _layer(lib, n_q_heads=32, n_kv_heads=8, head_dim=128, block=16, capacity=4160,
+               max_len_hint=4096)
+    f = lib.lib().orthrus_ar_verify_attend
+    assert f(ctypes.byref(L), None, 0x5000, 0x6000, 0x7000, 0x8000, 1 << 30, None) == 1
+    assert f(ctypes.byref(L), 0x4000, 0x5000, 0x6000, 0x7000, 0x8000, 256, None) == 4
+    assert f(None, 0x4000, 0x5000, 0x6000, 0x7000, 0x8000, 256, None) == 1
+    g = lib.lib().orthrus_consensus_accept
+    assert g(0x1000, 0, 0x2000, 1, 8, 1000, 0x3000, 0x4000, 0x5000, 0x6000, 0x7000, 8, None) == 4
+    assert g(0x1000, 3, 0x2000, 1, 8, 1000, 0x3000, 0x4000, 0x5000, 0x6000, 0x7000, 1 << 20, None) == 2
+    assert g(None, 0, 0x2000, 1, 8, 1000, 0x3000, 0x4000, 0x5000, 0x6000, 0x7000, 1 << 20, None) == 1
+    a = lib.lib().orthrus_kv_append
+    assert a(ctypes.byref(L), None, 0x2000, 0x3000, 1, None, 0, None) == 1
+    assert lib.lib().orthrus_set_path(b"bogus") == 1
+    assert lib.lib().orthrus_set_path(b"auto") == 0
