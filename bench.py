@@ -1,0 +1,484 @@
+#!/usr/bin/env python
+"""Benchmark of the Orthrus generation-step hot path on B200.
+
+One step = one full pass of the hot path over one batch of synthetic input:
+for every layer the diffusion-view block attention and the AR-view verify
+attention over the shared prefix KV cache, then the greedy consensus over the AR
+logits, then the commit of the accepted AR-view KV rows to every layer's cache.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME]
+  python bench.py --impl reference ...      # the CPU oracle on a bounded sample
+
+Prints one JSON line (rank 0).  With N > 1 (launched by torch.distributed.run) each
+rank runs an independent replica of the workload on its own GPU: the path has no
+exchange step, so there is no data-path collective ("replicas only", weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2605_12825_b200 import workloads as W  # noqa: E402
+
+DEFAULT_WORKLOAD = "cfg2_8b_b1"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+# ----------------------------------------------------------------------------- helpers
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def recorded_traffic(workload: str):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f).get(workload)
+    except Exception:
+        return None
+
+
+def attend_bytes(wl: W.Workload, lens) -> int:
+    """Algorithmic bytes of ONE attention call (one layer, one view): every prefix K
+    and V row once, the block K/V, the queries and the outputs."""
+    es = 2 if wl.dtype == "bf16" else 4
+    d = wl.head_dim
+    prefix = sum(int(p) for p in lens) * wl.n_kv_heads * 2 * d * es
+    blk = wl.batch * wl.block * wl.n_kv_heads * 2 * d * es
+    qo = wl.batch * wl.block * wl.n_q_heads * d * es * 2
+    return prefix + blk + qo
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- GPU arm
+
+class DeviceState:
+    """All tensors of the workload on one GPU, one set per layer (layers are distinct
+    buffers, so every timed read of a long-prefix workload misses L2)."""
+
+    def __init__(self, wl: W.Workload, layers: int, dev: torch.device):
+        from paper_2605_12825_b200 import binding as B
+        self.B, self.wl, self.layers, self.dev = B, wl, layers, dev
+        self.lens_host = W.prefix_lengths(wl)
+        self.cache_len = self.lens_host.to(dev)
+        self.cache_len0 = self.lens_host.to(dev)
+        self.host, self.t, self.layer, self.out_d, self.out_a = [], [], [], [], []
+        max_hint = int(self.lens_host.max())
+        for l in range(layers):
+            h = W.attention_inputs(wl, layer=l)
+            h.pop("cache_len")
+            t = {k: v.to(dev) for k, v in h.items()}
+            self.t.append(t)
+            self.host.append({k: v.pin_memory() for k, v in h.items() if "cache" not in k})
+            self.layer.append(B.make_layer(t["k_cache"], t["v_cache"], self.cache_len,
+                                           wl.n_q_heads, wl.block, max_hint))
+            self.out_d.append(torch.empty_like(t["q_diff"]))
+            self.out_a.append(torch.empty_like(t["q_ar"]))
+        self.ws = B.new_workspace(B.orthrus_attend_workspace_bytes(self.layer[0]))
+        lg = W.logits(wl)
+        greedy = lg.float().argmax(-1)          # input synthesis only: plants the agreement rate
+        self.logits_host = lg.pin_memory()
+        self.draft_host = W.drafts(wl, greedy).pin_memory()
+        self.logits = lg.to(dev)
+        self.draft = self.draft_host.to(dev)
+        Bn, K = wl.batch, wl.block
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.n_commit = torch.zeros(Bn, **i32)
+        self.committed = torch.zeros(Bn, K, **i32)
+        self.ar_argmax = torch.zeros(Bn, K, **i32)
+        self.next_anchor = torch.zeros(Bn, **i32)
+        self.cws = B.new_workspace(B.orthrus_consensus_workspace_bytes(Bn, K, wl.vocab))
+        self.res_host = torch.zeros(Bn, dtype=torch.int32).pin_memory()
+        self.out_host = [torch.empty(t["q_diff"].shape, dtype=t["q_diff"].dtype).pin_memory()
+                         for t in self.t[:1]]
+
+    # the four phases of a step, each a sequence of C-ABI calls on the current stream
+    def phase_diffusion(self):
+        B = self.B
+        for l in range(self.layers):
+            t = self.t[l]
+            B.orthrus_diffusion_block_attend(self.layer[l], t["q_diff"], t["k_diff_blk"],
+                                             t["v_diff_blk"], self.out_d[l], self.ws)
+
+    def phase_ar(self):
+        B = self.B
+        for l in range(self.layers):
+            t = self.t[l]
+            B.orthrus_ar_verify_attend(self.layer[l], t["q_ar"], t["k_ar_blk"], t["v_ar_blk"],
+                                       self.out_a[l], self.ws)
+
+    def phase_consensus(self):
+        self.B.orthrus_consensus_accept(self.logits, self.draft, self.n_commit, self.committed,
+                                        self.ar_argmax, self.next_anchor, self.cws)
+
+    def phase_commit(self):
+        B = self.B
+        for l in range(self.layers):
+            t = self.t[l]
+            # all layers share one length array: only the last call grows it
+            B.orthrus_kv_append(self.layer[l], t["k_ar_blk"], t["v_ar_blk"], self.n_commit,
+                                l == self.layers - 1, self.ws)
+        # the next step starts from the same prefix again (the appended bytes are identical
+        # every step, so this rewinds the state exactly)
+        self.cache_len.copy_(self.cache_len0)
+
+    def phases(self):
+        return [self.phase_diffusion, self.phase_ar, self.phase_consensus, self.phase_commit]
+
+    def h2d_inputs(self):
+        """End-to-end arm: this step's inputs come from pinned host memory."""
+        n = 0
+        for l in range(self.layers):
+            for k, hv in self.host[l].items():
+                self.t[l][k].copy_(hv, non_blocking=True)
+                n += hv.numel() * hv.element_size()
+        self.logits.copy_(self.logits_host, non_blocking=True)
+        self.draft.copy_(self.draft_host, non_blocking=True)
+        return n + self.logits_host.numel() * self.logits_host.element_size() + \
+            self.draft_host.numel() * 4
+
+    def d2h_results(self):
+        self.res_host.copy_(self.n_commit, non_blocking=True)
+        self.out_host[0].copy_(self.out_a[self.layers - 1], non_blocking=True)
+        return self.res_host.numel() * 4 + self.out_host[0].numel() * self.out_host[0].element_size()
+
+
+def capture(fn, stream):
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        fn()
+    return g
+
+
+def run_gpu(args):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (there is no CPU fallback for the GPU arm)")
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    from paper_2605_12825_b200 import build
+    if rank == 0:
+        build.build()
+    if dist is not None:
+        dist.barrier()
+    from paper_2605_12825_b200 import binding as B
+
+    wl = W.CONFIGS[args.workload]
+    layers = args.layers or wl.layers
+    st = DeviceState(wl, layers, dev)
+    stream = torch.cuda.Stream(device=dev)
+    phases = st.phases()
+
+    with torch.cuda.stream(stream):
+        for _ in range(2):                      # eager warm-up (sets kernel attributes)
+            for ph in phases:
+                ph()
+        stream.synchronize()
+        n0 = B.orthrus_launch_count()
+        for ph in phases:
+            ph()
+        launches_per_step = B.orthrus_launch_count() - n0
+        stream.synchronize()
+        graphs = None
+        if not args.no_graph:
+            graphs = [capture(ph, stream) for ph in phases]
+
+        def step(events=None):
+            for i in range(4):
+                if events is not None:
+                    events[i].record(stream)
+                if graphs is not None:
+                    graphs[i].replay()
+                else:
+                    phases[i]()
+            if events is not None:
+                events[4].record(stream)
+
+        for _ in range(max(args.warmup, 3)):
+            step()
+        stream.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+        sampler = ClockSampler(local)
+        sampler.start()
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+        for s in range(args.steps):
+            step(evs[s])
+        stream.synchronize()
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        if dist is not None:
+            dist.barrier()
+
+        total_ms = evs[0][0].elapsed_time(evs[-1][4])
+        phase_ms = [statistics.mean(e[i].elapsed_time(e[i + 1]) for e in evs) for i in range(4)]
+        n_commit = st.n_commit.cpu()
+        status = B.orthrus_read_status(st.ws, stream)
+
+        # end-to-end arm: host buffers in, results out, every step
+        for _ in range(2):
+            st.h2d_inputs(); step(); st.d2h_results()
+        stream.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e2e_steps = max(3, min(args.steps, 20))
+        e0.record(stream)
+        for _ in range(e2e_steps):
+            h2d = st.h2d_inputs()
+            step()
+            d2h = st.d2h_results()
+        e1.record(stream)
+        stream.synchronize()
+        e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    if status != 0:
+        raise SystemExit(f"bench.py: device status word {status} after the timed region")
+
+    ms_per_step = total_ms / args.steps
+    if dist is not None:
+        tt = torch.tensor([ms_per_step, e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_per_step, e2e_ms = float(tt[0]), float(tt[1])
+
+    call_bytes = attend_bytes(wl, st.lens_host)
+    step_bytes = call_bytes * 2 * layers
+    kv_gbs = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    tokens = int(n_commit.sum())
+    peak, peak_kind = measured_peak()
+    attend_ms = (phase_ms[0] + phase_ms[1]) / (2 * layers)
+    achieved = call_bytes / (attend_ms * 1e-3) / 1e9
+    path = B.orthrus_last_path()
+
+    out = {
+        "metric": "dual-view block-attention KV GB/s",
+        "value": round(kv_gbs, 2), "unit": "GB/s",
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.batch, "q_heads": wl.n_q_heads,
+                   "kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "block": wl.block,
+                   "prefix": [wl.prefix_min, wl.prefix_max], "vocab": wl.vocab, "layers": layers,
+                   "step": "layers x (diffusion attend + AR verify attend) + consensus + "
+                           "layers x KV commit (+ rewind of cache_len)",
+                   "l2": "inputs larger than L2 (distinct KV per layer)" if step_bytes > 2.5e8
+                         else "L2-resident (reported, not a roofline workload)",
+                   "cuda_graph": not args.no_graph, "attend_path": path,
+                   "multi_gpu": "replicas only"},
+        "pct_of_hbm_peak": {"of_measured_%.0f" % peak if peak_kind == "measured" else
+                            "of_fallback_%.0f" % peak: round(100 * kv_gbs / world / peak, 2),
+                            "of_nominal_8000": round(100 * kv_gbs / world / NOMINAL_HBM_GBS, 2)},
+        "verified_tokens_per_s": round(world * tokens / (ms_per_step * 1e-3), 1),
+        "verified_tokens_per_step": tokens,
+        "tokens_per_forward_pass": round(tokens / wl.batch / 2.0, 4),
+        "phase_ms": {"diffusion_attend": round(phase_ms[0], 5), "ar_verify_attend": round(phase_ms[1], 5),
+                     "consensus": round(phase_ms[2], 5), "kv_commit": round(phase_ms[3], 5)},
+        "gpu_launches": int(launches_per_step * args.steps),
+        "clocks": clocks,
+        "e2e": {"value": round(world * step_bytes / (e2e_ms * 1e-3) / 1e9, 2), "unit": "GB/s",
+                "ms_per_step": round(e2e_ms, 5), "h2d_bytes_per_step": int(h2d),
+                "d2h_bytes_per_step": int(d2h),
+                "note": "per-step inputs (Q, block KV, logits, drafts) from pinned host memory; "
+                        "the prefix KV cache is resident state"},
+        "roofline": {"bound": "hbm", "kernel": f"block attention ({path}) + split merge, per call",
+                     "achieved": round(achieved, 2), "peak": peak, "peak_kind": peak_kind,
+                     "unit": "GB/s", "frac": round(achieved / peak, 4),
+                     "algorithmic_bytes_per_launch": call_bytes,
+                     "avg_launch_us": round(attend_ms * 1e3, 3),
+                     "traffic": recorded_traffic(wl.name)},
+    }
+    if rank == 0:
+        if not args.no_cpu_baseline and world == 1:
+            out["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_budget)
+        print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- oracle arm
+
+def oracle_sample(wl: W.Workload, layer: int = 0):
+    """A bounded sample of the workload for the CPU oracle: one layer, both views, as
+    many query rows (spread over all sequences) as cost about what one full layer of
+    the 8B single-sequence workload costs, plus consensus and commit."""
+    t = W.attention_inputs(wl, layer=layer)
+    B_, K, Hq = wl.batch, wl.block, wl.n_q_heads
+    g = torch.Generator().manual_seed(1)
+    mean_len = float(t["cache_len"].double().mean()) + K
+    n_rows = int(512 * 4112 * 128 / (mean_len * wl.head_dim))
+    n_rows = max(1, min(n_rows, B_ * K * Hq))
+    flat = torch.randperm(B_ * K * Hq, generator=g)[:n_rows]
+    rows = torch.stack([flat // (K * Hq), (flat // Hq) % K, flat % Hq], dim=1).to(torch.int32)
+    lg = W.logits(wl)
+    return t, rows, lg
+
+
+def oracle_step(wl, t, rows, lg):
+    import oracle
+    oracle.block_attend_rows(oracle.VIEW_DIFFUSION, rows, t["q_diff"], t["k_diff_blk"],
+                             t["v_diff_blk"], t["k_cache"], t["v_cache"], t["cache_len"])
+    oracle.block_attend_rows(oracle.VIEW_AR, rows, t["q_ar"], t["k_ar_blk"], t["v_ar_blk"],
+                             t["k_cache"], t["v_cache"], t["cache_len"])
+    draft = torch.zeros(wl.batch, wl.block, dtype=torch.int32)
+    n, *_ = oracle.consensus_accept(lg, draft)
+    lens = t["cache_len"].clone()
+    oracle.kv_append(t["k_cache"], t["v_cache"], lens, t["k_ar_blk"], t["v_ar_blk"], n)
+
+
+def sample_bytes(wl, t, rows):
+    """Algorithmic KV bytes credited to the sample: the oracle streams the prefix of a
+    row's KV head once per sampled row (it has no reuse), so the rows' share of one
+    layer's two attention calls is credited."""
+    full = attend_bytes(wl, t["cache_len"]) * 2
+    return full * rows.shape[0] / (wl.batch * wl.block * wl.n_q_heads)
+
+
+def cpu_baseline(wl, budget_s=20.0):
+    """Times the oracle, as it stands, on samples of successive layers until about
+    `budget_s` core-seconds of CPU work have been spent."""
+    import oracle
+    oracle.build()
+    cores = oracle.num_threads()
+    spent, nbytes, layer, rows_n = 0.0, 0.0, 0, 0
+    lg = W.logits(wl)
+    while spent * cores < budget_s and layer < max(wl.layers, 8):
+        t, rows, _ = oracle_sample(wl, layer)
+        t0 = time.perf_counter()
+        oracle_step(wl, t, rows, lg)
+        spent += time.perf_counter() - t0
+        nbytes += sample_bytes(wl, t, rows)
+        rows_n = rows.shape[0]
+        layer += 1
+    return {"value": round(nbytes / spent / 1e9, 4), "unit": "GB/s", "cores": cores,
+            "kind": "oracle", "seconds": round(spent, 3),
+            "sample": f"{wl.name}: {layer} layer(s), both views, {rows_n} of "
+                      f"{wl.batch * wl.block * wl.n_q_heads} query rows per layer, each with a "
+                      f"full consensus and commit"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    wl = W.CONFIGS[args.workload]
+    t, rows, lg = oracle_sample(wl)
+    for _ in range(args.warmup):
+        oracle_step(wl, t, rows, lg)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(wl, t, rows, lg)
+    dt = (time.perf_counter() - t0) / args.steps
+    val = round(sample_bytes(wl, t, rows) / dt / 1e9, 4)
+    sample = (f"{wl.name}: 1 layer, both views, {rows.shape[0]} of "
+              f"{wl.batch * wl.block * wl.n_q_heads} query rows, + full consensus and commit")
+    print(json.dumps({
+        "impl": "reference", "metric": "dual-view block-attention KV GB/s", "value": val,
+        "unit": "GB/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": oracle.num_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.CONFIGS))
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count")
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=20.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()
