@@ -73,12 +73,12 @@ struct Plan { int chunk, n_splits; };
 
 static Plan make_plan(const orthrus_layer_t *L)
 {
-    const int tile = 64;
+    const int tile = 128;
     const int units = L->batch * L->n_kv_heads;
     const int max_len = max_len_of(L);
     const int tiles = max_len > 0 ? (max_len + tile - 1) / tile : 1;
     const int target = env_int("ORTHRUS_TARGET_CTAS", 2 * kNumSMs);
-    const int min_chunk_tiles = env_int("ORTHRUS_MIN_CHUNK_TILES", 4);
+    const int min_chunk_tiles = env_int("ORTHRUS_MIN_CHUNK_TILES", 2);
     int splits = (target + units - 1) / units;
     const int forced = env_int("ORTHRUS_SPLITS", 0);
     if (forced > 0) splits = forced;
@@ -139,7 +139,10 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const int want = current_path();
     cudaError_t e;
-    if (want != PATH_SIMT && mma_path_supports(p, L->dtype)) {
+    if ((want == PATH_AUTO || want == PATH_TCGEN05) && tc_path_supports(p, L->dtype)) {
+        t_last_path = "tcgen05";
+        e = launch_attend_tc(p, cs);
+    } else if (want != PATH_SIMT && mma_path_supports(p, L->dtype)) {
         t_last_path = "mma";
         e = launch_attend_mma(p, cs);
     } else {

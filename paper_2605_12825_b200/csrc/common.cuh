@@ -53,6 +53,8 @@ cudaError_t launch_attend_simt(const AttnParams &p, int dtype, cudaStream_t st);
 bool mma_path_supports(const AttnParams &p, int dtype);
 cudaError_t launch_attend_mma(const AttnParams &p, cudaStream_t st);
 int mma_tile_positions();
+bool tc_path_supports(const AttnParams &p, int dtype);
+cudaError_t launch_attend_tc(const AttnParams &p, cudaStream_t st);
 cudaError_t launch_combine(const AttnParams &p, int dtype, cudaStream_t st);
 
 cudaError_t launch_consensus(const void *logits, int dtype, const int32_t *draft, int B, int K,

@@ -13,16 +13,26 @@ from _gpu_util import (assert_close, oracle_attend, run_attend, small_workload)
 pytestmark = pytest.mark.gpu
 VIEWS = [oracle.VIEW_DIFFUSION, oracle.VIEW_AR]
 NAN = float("nan")
+PATHS = ["simt", "mma", "tcgen05"]
+
+
+def taken(path, wl):
+    """The path a request resolves to: tcgen05 needs head_dim 128, mma needs 64 or 128."""
+    if path == "tcgen05" and wl.head_dim != 128:
+        path = "mma"
+    if path == "mma" and wl.head_dim not in (64, 128):
+        path = "simt"
+    return path
 
 
 @pytest.mark.parametrize("view", VIEWS)
 @pytest.mark.parametrize("P", [0, 1, 3, 17, 63, 64, 65, 130, 257])
-@pytest.mark.parametrize("path", ["simt", "mma"])
+@pytest.mark.parametrize("path", PATHS)
 def test_tiny_prefixes_bf16(view, P, path):
     wl = small_workload(2, 8, 8, 2, 64, P, P, std=0.5)
     t = W.attention_inputs(wl, fill_tail=NAN)
     got, status, used = run_attend(view, t, wl, path=path)
-    assert status == 0 and used == path
+    assert status == 0 and used == taken(path, wl)
     assert_close(got, oracle_attend(view, t), torch.bfloat16, f"P={P}")
 
 
@@ -37,12 +47,12 @@ def test_tiny_prefixes_bf16(view, P, path):
     (2, 64, 2, 2, 128, 10, 90),        # widest block
     (1, 5, 6, 2, 64, 77, 77),          # M = 15, not a multiple of anything
 ])
-@pytest.mark.parametrize("path", ["simt", "mma"])
+@pytest.mark.parametrize("path", PATHS)
 def test_shapes_bf16(view, shape, path):
     wl = small_workload(*shape, std=0.7)
     t = W.attention_inputs(wl, fill_tail=NAN)
     got, status, used = run_attend(view, t, wl, path=path)
-    assert status == 0 and used == path
+    assert status == 0 and used == taken(path, wl)
     assert_close(got, oracle_attend(view, t), torch.bfloat16, str(shape))
 
 
@@ -69,7 +79,7 @@ def test_fp32_mode(view, shape):
 
 @pytest.mark.parametrize("view", VIEWS)
 @pytest.mark.parametrize("splits", [1, 2, 3, 7])
-@pytest.mark.parametrize("path", ["simt", "mma"])
+@pytest.mark.parametrize("path", PATHS)
 def test_forced_splits_agree(view, splits, path):
     """Split-KV with empty, partial and full splits (ragged batch) gives the same result."""
     wl = small_workload(3, 16, 8, 2, 128, 1, 900, std=0.7)
@@ -80,7 +90,7 @@ def test_forced_splits_agree(view, splits, path):
 
 
 @pytest.mark.parametrize("view", VIEWS)
-@pytest.mark.parametrize("path", ["simt", "mma"])
+@pytest.mark.parametrize("path", PATHS)
 def test_peaked_scores(view, path):
     """Queries scaled x16: the softmax is dominated by a few keys, so wrong masks or
     a wrong running max show up at full magnitude."""
@@ -91,7 +101,7 @@ def test_peaked_scores(view, path):
     assert_close(got, oracle_attend(view, t), torch.bfloat16)
 
 
-@pytest.mark.parametrize("path", ["simt", "mma"])
+@pytest.mark.parametrize("path", PATHS)
 def test_planted_key_hidden_by_the_causal_rule(path):
     """A block key with an overwhelming score: every diffusion row collapses onto its
     value row, AR rows before it must not see it at all."""
