@@ -67,36 +67,57 @@ static int max_len_of(const orthrus_layer_t *L)
     return L->max_len_hint > 0 ? L->max_len_hint : (int)(L->capacity - L->block);
 }
 
-// Split-KV plan: a pure function of the descriptor (and of two tuning variables read
-// from the environment), so that the workspace query and the launch always agree.
-struct Plan { int chunk, n_splits; };
+// Split-KV plan: a pure function of the descriptor, the kernel path and a few tuning
+// variables read from the environment, so that the workspace query and the launch agree.
+struct Plan { int chunk, n_splits, tile; };
 
-static Plan make_plan(const orthrus_layer_t *L)
+static bool tc_shape(const orthrus_layer_t *L)
 {
-    const int tile = 128;
+    return L->dtype == ORTHRUS_BF16 && L->head_dim == 128 && L->block <= 64;
+}
+
+static Plan make_plan(const orthrus_layer_t *L, bool tc)
+{
+    const int granule = tc ? 64 : 128;
     const int units = L->batch * L->n_kv_heads;
+    const int M = (L->n_q_heads / L->n_kv_heads) * L->block;
+    const int row_tiles = tc ? (M + 127) / 128 : 1;
     const int max_len = max_len_of(L);
-    const int tiles = max_len > 0 ? (max_len + tile - 1) / tile : 1;
-    const int target = env_int("ORTHRUS_TARGET_CTAS", 2 * kNumSMs);
+    const int tiles = max_len > 0 ? (max_len + granule - 1) / granule : 1;
+    const int target = env_int("ORTHRUS_TARGET_CTAS", tc ? kNumSMs : 2 * kNumSMs);
     const int min_chunk_tiles = env_int("ORTHRUS_MIN_CHUNK_TILES", 2);
-    int splits = (target + units - 1) / units;
+    int splits = (target + units * row_tiles - 1) / (units * row_tiles);
     const int forced = env_int("ORTHRUS_SPLITS", 0);
     if (forced > 0) splits = forced;
-    int max_splits = tiles / min_chunk_tiles;
-    if (forced > 0) max_splits = tiles;
+    int max_splits = forced > 0 ? tiles : tiles / min_chunk_tiles;
     if (max_splits < 1) max_splits = 1;
     if (max_splits > kMaxSplits) max_splits = kMaxSplits;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
+    if (tc && splits <= 16 && forced == 0) {
+        // the splits of a unit form one thread-block cluster: keep its size a power of two
+        int p2 = 1;
+        while (p2 * 2 <= splits) p2 *= 2;
+        if (p2 < splits && p2 * 2 <= max_splits && p2 * 2 <= 16) p2 *= 2;
+        splits = p2;
+    }
     const int chunk_tiles = (tiles + splits - 1) / splits;
     Plan pl;
-    pl.chunk = chunk_tiles * tile;
+    pl.chunk = chunk_tiles * granule;
     pl.n_splits = max_len > 0 ? (max_len + pl.chunk - 1) / pl.chunk : 1;
+    if (tc && forced == 0 && pl.n_splits <= 16) {       // grid extent = cluster size = power of two
+        int p2 = 1;
+        while (p2 < pl.n_splits) p2 *= 2;
+        pl.n_splits = p2;
+    }
+    const int tn = env_int("ORTHRUS_TC_TN", pl.chunk <= 512 ? 64 : 128);
+    pl.tile = tc ? (tn == 64 ? 64 : 128) : granule;
     return pl;
 }
 
-static size_t partial_bytes(const orthrus_layer_t *L, const Plan &pl, size_t *ml_off)
+static size_t partial_bytes(const orthrus_layer_t *L, const Plan &pl, size_t *ml_off, bool tc = false)
 {
+    if (tc && tc_cluster_for_splits(pl.n_splits) == pl.n_splits) { if (ml_off) *ml_off = 0; return 0; }
     const size_t units = (size_t)L->batch * L->n_kv_heads;
     const size_t M = (size_t)(L->n_q_heads / L->n_kv_heads) * L->block;
     if (pl.n_splits == 1) { if (ml_off) *ml_off = 0; return 0; }
@@ -118,9 +139,11 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
         !aligned16(ws) || !aligned16(L->k_cache) || !aligned16(L->v_cache) ||
         (reinterpret_cast<uintptr_t>(L->cache_len) & 3))
         return ORTHRUS_ERR_INVALID_ARG;
-    const Plan pl = make_plan(L);
+    const int want = current_path();
+    const bool tc = (want == PATH_AUTO || want == PATH_TCGEN05) && tc_shape(L);
+    const Plan pl = make_plan(L, tc);
     size_t ml_off = 0;
-    const size_t need = kHeaderBytes + partial_bytes(L, pl, &ml_off);
+    const size_t need = kHeaderBytes + partial_bytes(L, pl, &ml_off, tc);
     if (ws_bytes < need) return ORTHRUS_ERR_WORKSPACE;
 
     AttnParams p;
@@ -137,11 +160,14 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
     p.scale_log2 = scale * 1.4426950408889634f;
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    const int want = current_path();
     cudaError_t e;
-    if ((want == PATH_AUTO || want == PATH_TCGEN05) && tc_path_supports(p, L->dtype)) {
+    bool merge_kernel = pl.n_splits > 1;
+    if (tc && tc_path_supports(p, L->dtype)) {
         t_last_path = "tcgen05";
-        e = launch_attend_tc(p, cs);
+        e = launch_attend_tc(p, pl.tile, cs);
+        merge_kernel = tc_cluster_for_splits(pl.n_splits) != pl.n_splits;
+    } else if (tc) {
+        return ORTHRUS_ERR_CUDA;            // the driver offers no tensor-map encoder
     } else if (want != PATH_SIMT && mma_path_supports(p, L->dtype)) {
         t_last_path = "mma";
         e = launch_attend_mma(p, cs);
@@ -150,7 +176,7 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
         e = launch_attend_simt(p, L->dtype, cs);
     }
     if (e != cudaSuccess) return ORTHRUS_ERR_CUDA;
-    if (pl.n_splits > 1) {
+    if (merge_kernel) {
         e = launch_combine(p, L->dtype, cs);
         if (e != cudaSuccess) return ORTHRUS_ERR_CUDA;
     }
@@ -166,7 +192,13 @@ extern "C" {
 size_t orthrus_attend_workspace_bytes(const orthrus_layer_t *layer)
 {
     if (check_layer(layer) != ORTHRUS_OK) return 0;
-    return kHeaderBytes + partial_bytes(layer, make_plan(layer), nullptr);
+    // enough for whichever kernel path a later call resolves to
+    size_t need = partial_bytes(layer, make_plan(layer, false), nullptr, false);
+    if (tc_shape(layer)) {
+        const size_t n2 = partial_bytes(layer, make_plan(layer, true), nullptr, true);
+        if (n2 > need) need = n2;
+    }
+    return kHeaderBytes + need;
 }
 
 orthrus_status_t orthrus_workspace_init(void *workspace, size_t workspace_bytes, void *stream)

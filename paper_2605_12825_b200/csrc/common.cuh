@@ -54,7 +54,8 @@ bool mma_path_supports(const AttnParams &p, int dtype);
 cudaError_t launch_attend_mma(const AttnParams &p, cudaStream_t st);
 int mma_tile_positions();
 bool tc_path_supports(const AttnParams &p, int dtype);
-cudaError_t launch_attend_tc(const AttnParams &p, cudaStream_t st);
+cudaError_t launch_attend_tc(const AttnParams &p, int tile, cudaStream_t st);
+int tc_cluster_for_splits(int n_splits);
 cudaError_t launch_combine(const AttnParams &p, int dtype, cudaStream_t st);
 
 cudaError_t launch_consensus(const void *logits, int dtype, const int32_t *draft, int B, int K,
