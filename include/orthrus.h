@@ -78,12 +78,35 @@ typedef struct {
     int32_t max_len_hint;   /* host upper bound on every P_b; sizes the split-KV
                                grid.  0 means capacity - block                      */
     float softmax_scale;    /* 0 selects 1/sqrt(head_dim), the scale of Eq. 4       */
+    uint32_t flags;         /* OR of ORTHRUS_LAYER_* bits, 0 for none               */
 } orthrus_layer_t;
+
+/*
+ * orthrus_layer_t.flags
+ *
+ * ORTHRUS_LAYER_CACHE_QUIESCENT: a promise by the caller that the kernel enqueued
+ * immediately before this call on the same stream writes neither cache_len nor any
+ * cache row below cache_len (in a generation loop that kernel is the projection that
+ * produced q and the block KV; the cache was last written by the previous cycle's
+ * commit).  The attention kernels are launched with programmatic stream
+ * serialisation: they may start while the preceding kernel is still running and wait
+ * for it on the device before touching anything it may have produced.  With this
+ * flag they request the first prefix K/V tiles before that wait.  Without it nothing
+ * is read early and any caller is safe.
+ *
+ * ORTHRUS_LAYER_NO_EARLY_LAUNCH: launch with ordinary stream order only.
+ */
+enum {
+    ORTHRUS_LAYER_CACHE_QUIESCENT = 1,
+    ORTHRUS_LAYER_NO_EARLY_LAUNCH = 2
+};
 
 /*
  * Bytes of workspace the two attention calls (and orthrus_kv_append) need for
  * this layer shape: a 256-byte header holding the status word, followed by the
- * split-KV partial results.  Returns 0 for an invalid descriptor.
+ * split-KV partial results of the kernel paths that keep them in global memory
+ * (the tcgen05 path merges its splits on chip and uses the header only).
+ * Returns 0 for an invalid descriptor.
  */
 size_t orthrus_attend_workspace_bytes(const orthrus_layer_t *layer);
 
@@ -147,6 +170,20 @@ orthrus_status_t orthrus_consensus_accept(const void *ar_logits, int32_t dtype,
 orthrus_status_t orthrus_kv_append(const orthrus_layer_t *layer, const void *k_ar_blk,
         const void *v_ar_blk, const int32_t *n_commit, int32_t update_len,
         void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The same commit for n_layers layers in one launch: the cycle's verify pass has
+ * produced the AR-view block KV of every layer by the time the consensus is known, so
+ * one kernel moves all of it.  layers[l] is the l-th layer's descriptor (a HOST array;
+ * all layers must agree in batch, n_kv_heads, head_dim, block, dtype and capacity);
+ * k_ar_blks[l] / v_ar_blks[l] are HOST arrays of DEVICE pointers to that layer's
+ * [B][K][Hkv][d] block tensors.  With update_len != 0 every DISTINCT cache_len array
+ * among the layers grows by n_commit once, after all of its layers have been copied
+ * (layers sharing one array are bumped once).  1 <= n_layers <= 128.
+ */
+orthrus_status_t orthrus_kv_append_layers(const orthrus_layer_t *layers, int32_t n_layers,
+        const void *const *k_ar_blks, const void *const *v_ar_blks, const int32_t *n_commit,
+        int32_t update_len, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * Copies the device status word to *host_status and waits for the stream (the

@@ -24,7 +24,7 @@ EXPORTS = [
     "orthrus_attend_workspace_bytes", "orthrus_workspace_init",
     "orthrus_diffusion_block_attend", "orthrus_ar_verify_attend",
     "orthrus_consensus_workspace_bytes", "orthrus_consensus_accept",
-    "orthrus_kv_append", "orthrus_read_status", "orthrus_set_path", "orthrus_last_path",
+    "orthrus_kv_append", "orthrus_kv_append_layers", "orthrus_read_status", "orthrus_set_path", "orthrus_last_path",
     "orthrus_launch_count", "orthrus_status_string", "orthrus_version",
 ]
 
@@ -43,7 +43,11 @@ class Layer(ctypes.Structure):
                 ("block", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("capacity", ctypes.c_int64), ("k_cache", ctypes.c_void_p),
                 ("v_cache", ctypes.c_void_p), ("cache_len", ctypes.c_void_p),
-                ("max_len_hint", ctypes.c_int32), ("softmax_scale", ctypes.c_float)]
+                ("max_len_hint", ctypes.c_int32), ("softmax_scale", ctypes.c_float),
+                ("flags", ctypes.c_uint32)]
+
+
+LAYER_CACHE_QUIESCENT, LAYER_NO_EARLY_LAUNCH = 1, 2
 
 
 def _load() -> ctypes.CDLL:
@@ -68,6 +72,9 @@ def _load() -> ctypes.CDLL:
     lib.orthrus_consensus_accept.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.orthrus_kv_append.restype = ctypes.c_int
     lib.orthrus_kv_append.argtypes = [LP, vp, vp, vp, i32, vp, sz, vp]
+    lib.orthrus_kv_append_layers.restype = ctypes.c_int
+    lib.orthrus_kv_append_layers.argtypes = [LP, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, i32,
+                                             vp, sz, vp]
     lib.orthrus_read_status.restype = ctypes.c_int
     lib.orthrus_read_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     lib.orthrus_set_path.restype = ctypes.c_int
@@ -112,12 +119,12 @@ def _check(code: int, where: str) -> None:
 
 def make_layer(k_cache: torch.Tensor, v_cache: torch.Tensor, cache_len: torch.Tensor,
                n_q_heads: int, block: int, max_len_hint: int = 0,
-               softmax_scale: float = 0.0) -> Layer:
+               softmax_scale: float = 0.0, flags: int = 0) -> Layer:
     """Describe one layer's shared cache ([B][Hkv][capacity][d]) and block shape."""
     B, Hkv, cap, d = k_cache.shape
     return Layer(B, n_q_heads, Hkv, d, block, dtype_code(k_cache.dtype), cap,
                  k_cache.data_ptr(), v_cache.data_ptr(), cache_len.data_ptr(),
-                 max_len_hint, softmax_scale)
+                 max_len_hint, softmax_scale, flags)
 
 
 def orthrus_attend_workspace_bytes(layer: Layer) -> int:
@@ -168,6 +175,18 @@ def orthrus_kv_append(layer: Layer, k_ar_blk, v_ar_blk, n_commit, update_len: bo
         ctypes.byref(layer), _ptr(k_ar_blk), _ptr(v_ar_blk), _ptr(n_commit),
         1 if update_len else 0, _ptr(workspace), 0 if workspace is None else workspace.numel(),
         _stream(stream)), "orthrus_kv_append")
+
+
+def orthrus_kv_append_layers(layers, k_ar_blks, v_ar_blks, n_commit, update_len: bool = True,
+                             workspace=None, stream=None) -> None:
+    """`layers`: sequence of Layer; `k_ar_blks` / `v_ar_blks`: one tensor per layer."""
+    n = len(layers)
+    arr = (Layer * n)(*layers)
+    kp = (ctypes.c_void_p * n)(*[t.data_ptr() for t in k_ar_blks])
+    vp = (ctypes.c_void_p * n)(*[t.data_ptr() for t in v_ar_blks])
+    _check(_lib.orthrus_kv_append_layers(
+        arr, n, kp, vp, _ptr(n_commit), 1 if update_len else 0, _ptr(workspace),
+        0 if workspace is None else workspace.numel(), _stream(stream)), "orthrus_kv_append_layers")
 
 
 def orthrus_read_status(workspace, stream=None) -> int:

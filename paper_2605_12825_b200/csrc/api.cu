@@ -59,6 +59,8 @@ static orthrus_status_t check_layer(const orthrus_layer_t *L)
     if (L->block > L->capacity) return ORTHRUS_ERR_CAPACITY;
     if (L->capacity > 0x7fffffffLL) return ORTHRUS_ERR_UNSUPPORTED;
     if ((long long)L->max_len_hint + L->block > L->capacity) return ORTHRUS_ERR_CAPACITY;
+    if (L->flags & ~(uint32_t)(ORTHRUS_LAYER_CACHE_QUIESCENT | ORTHRUS_LAYER_NO_EARLY_LAUNCH))
+        return ORTHRUS_ERR_INVALID_ARG;
     return ORTHRUS_OK;
 }
 
@@ -73,54 +75,65 @@ struct Plan { int chunk, n_splits, tile; };
 
 static bool tc_shape(const orthrus_layer_t *L)
 {
-    return L->dtype == ORTHRUS_BF16 && L->head_dim == 128 && L->block <= 64;
+    return L->dtype == ORTHRUS_BF16 && L->head_dim == 128 && L->block <= 64 &&
+           tc_row_tiles(L->n_q_heads / L->n_kv_heads, L->block) > 0;
 }
 
 static Plan make_plan(const orthrus_layer_t *L, bool tc)
 {
-    const int granule = tc ? 64 : 128;
-    const int units = L->batch * L->n_kv_heads;
-    const int M = (L->n_q_heads / L->n_kv_heads) * L->block;
-    const int row_tiles = tc ? (M + 127) / 128 : 1;
     const int max_len = max_len_of(L);
-    const int tiles = max_len > 0 ? (max_len + granule - 1) / granule : 1;
-    const int target = env_int("ORTHRUS_TARGET_CTAS", tc ? kNumSMs : 2 * kNumSMs);
-    const int min_chunk_tiles = env_int("ORTHRUS_MIN_CHUNK_TILES", 2);
-    int splits = (target + units * row_tiles - 1) / (units * row_tiles);
     const int forced = env_int("ORTHRUS_SPLITS", 0);
+    Plan pl;
+    if (tc) {
+        // The splits of a unit are the CTAs of one thread-block cluster (<= 16).  Few units:
+        // as many splits as still fit on the GPU in one wave.  Many units: enough CTAs for
+        // about three waves, so that sequences of unequal length pack well.
+        const int tn = tc_tile_positions();
+        const int units = L->batch * L->n_kv_heads * tc_row_tiles(L->n_q_heads / L->n_kv_heads, L->block);
+        const int slots = tc_ctas_per_sm() * kNumSMs;
+        const int tiles = max_len > 0 ? (max_len + tn - 1) / tn : 1;
+        int S = 1;
+        if (forced > 0) {
+            S = forced;
+        } else if (units * 2 <= slots) {
+            const int min_tiles = env_int("ORTHRUS_MIN_CHUNK_TILES", 2);
+            while (S < 16 && units * S * 2 <= slots && tiles / (S * 2) >= min_tiles) S *= 2;
+        } else {
+            while (S < 16 && units * S < 3 * slots && tiles / (S * 2) >= 8) S *= 2;
+        }
+        if (S > 16) S = 16;
+        if (S > tiles) S = tiles;
+        if (S < 1) S = 1;
+        pl.n_splits = S;
+        pl.chunk = ((tiles + S - 1) / S) * tn;
+        pl.tile = tn;
+        return pl;
+    }
+    const int granule = 128;
+    const int units = L->batch * L->n_kv_heads;
+    const int tiles = max_len > 0 ? (max_len + granule - 1) / granule : 1;
+    const int target = env_int("ORTHRUS_TARGET_CTAS", 2 * kNumSMs);
+    const int min_chunk_tiles = env_int("ORTHRUS_MIN_CHUNK_TILES", 2);
+    int splits = (target + units - 1) / units;
     if (forced > 0) splits = forced;
     int max_splits = forced > 0 ? tiles : tiles / min_chunk_tiles;
     if (max_splits < 1) max_splits = 1;
     if (max_splits > kMaxSplits) max_splits = kMaxSplits;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
-    if (tc && splits <= 16 && forced == 0) {
-        // the splits of a unit form one thread-block cluster: keep its size a power of two
-        int p2 = 1;
-        while (p2 * 2 <= splits) p2 *= 2;
-        if (p2 < splits && p2 * 2 <= max_splits && p2 * 2 <= 16) p2 *= 2;
-        splits = p2;
-    }
     const int chunk_tiles = (tiles + splits - 1) / splits;
-    Plan pl;
     pl.chunk = chunk_tiles * granule;
     pl.n_splits = max_len > 0 ? (max_len + pl.chunk - 1) / pl.chunk : 1;
-    if (tc && forced == 0 && pl.n_splits <= 16) {       // grid extent = cluster size = power of two
-        int p2 = 1;
-        while (p2 < pl.n_splits) p2 *= 2;
-        pl.n_splits = p2;
-    }
-    const int tn = env_int("ORTHRUS_TC_TN", pl.chunk <= 512 ? 64 : 128);
-    pl.tile = tc ? (tn == 64 ? 64 : 128) : granule;
+    pl.tile = granule;
     return pl;
 }
 
 static size_t partial_bytes(const orthrus_layer_t *L, const Plan &pl, size_t *ml_off, bool tc = false)
 {
-    if (tc && tc_cluster_for_splits(pl.n_splits) == pl.n_splits) { if (ml_off) *ml_off = 0; return 0; }
+    if (ml_off) *ml_off = 0;
+    if (tc || pl.n_splits == 1) return 0;      // the tcgen05 path merges its splits on chip
     const size_t units = (size_t)L->batch * L->n_kv_heads;
     const size_t M = (size_t)(L->n_q_heads / L->n_kv_heads) * L->block;
-    if (pl.n_splits == 1) { if (ml_off) *ml_off = 0; return 0; }
     const size_t o_bytes = units * pl.n_splits * M * L->head_dim * sizeof(float);
     const size_t ml_bytes = units * pl.n_splits * M * 2 * sizeof(float);
     if (ml_off) *ml_off = o_bytes;
@@ -164,8 +177,10 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
     bool merge_kernel = pl.n_splits > 1;
     if (tc && tc_path_supports(p, L->dtype)) {
         t_last_path = "tcgen05";
-        e = launch_attend_tc(p, pl.tile, cs);
-        merge_kernel = tc_cluster_for_splits(pl.n_splits) != pl.n_splits;
+        int flags = (int)(L->flags & (ORTHRUS_LAYER_CACHE_QUIESCENT | ORTHRUS_LAYER_NO_EARLY_LAUNCH));
+        if (env_int("ORTHRUS_NO_EARLY_LAUNCH", 0)) flags |= ORTHRUS_LAYER_NO_EARLY_LAUNCH;
+        e = launch_attend_tc(p, flags, cs);
+        merge_kernel = false;
     } else if (tc) {
         return ORTHRUS_ERR_CUDA;            // the driver offers no tensor-map encoder
     } else if (want != PATH_SIMT && mma_path_supports(p, L->dtype)) {
@@ -271,6 +286,42 @@ orthrus_status_t orthrus_kv_append(const orthrus_layer_t *layer, const void *k_a
     cudaError_t e = launch_kv_append(*layer, k_ar_blk, v_ar_blk, n_commit, update_len,
                                      static_cast<int32_t *>(workspace),
                                      static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+}
+
+orthrus_status_t orthrus_kv_append_layers(const orthrus_layer_t *layers, int32_t n_layers,
+        const void *const *k_ar_blks, const void *const *v_ar_blks, const int32_t *n_commit,
+        int32_t update_len, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!layers || !k_ar_blks || !v_ar_blks || !n_commit || n_layers < 1 || n_layers > 128)
+        return ORTHRUS_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(n_commit) & 3) return ORTHRUS_ERR_INVALID_ARG;
+    if (workspace && (workspace_bytes < (size_t)kHeaderBytes || !aligned16(workspace)))
+        return ORTHRUS_ERR_WORKSPACE;
+    AppendLayer al[128];
+    int32_t *lens[128];
+    int n_lens = 0;
+    const orthrus_layer_t &L0 = layers[0];
+    for (int l = 0; l < n_layers; ++l) {
+        const orthrus_layer_t &L = layers[l];
+        const orthrus_status_t st = check_layer(&L);
+        if (st != ORTHRUS_OK) return st;
+        if (L.batch != L0.batch || L.n_kv_heads != L0.n_kv_heads || L.head_dim != L0.head_dim ||
+            L.block != L0.block || L.dtype != L0.dtype || L.capacity != L0.capacity)
+            return ORTHRUS_ERR_INVALID_ARG;
+        if (!k_ar_blks[l] || !v_ar_blks[l] || !L.k_cache || !L.v_cache || !L.cache_len)
+            return ORTHRUS_ERR_INVALID_ARG;
+        if (!aligned16(k_ar_blks[l]) || !aligned16(v_ar_blks[l]) || !aligned16(L.k_cache) ||
+            !aligned16(L.v_cache) || (reinterpret_cast<uintptr_t>(L.cache_len) & 3))
+            return ORTHRUS_ERR_INVALID_ARG;
+        al[l] = AppendLayer{L.k_cache, L.v_cache, k_ar_blks[l], v_ar_blks[l], L.cache_len};
+        bool seen = false;
+        for (int j = 0; j < n_lens; ++j) seen |= lens[j] == L.cache_len;
+        if (!seen) lens[n_lens++] = L.cache_len;
+    }
+    cudaError_t e = launch_kv_append_layers(L0, al, n_layers, lens, update_len ? n_lens : 0, n_commit,
+                                            static_cast<int32_t *>(workspace),
+                                            static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
 }
 

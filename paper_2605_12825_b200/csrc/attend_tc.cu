@@ -1,30 +1,38 @@
 // Split-KV flash-decode block attention on the 5th-generation tensor cores
 // (tcgen05.mma with TMEM accumulators), bf16, head_dim 128, both views.
 //
-// One CTA streams one split of one (sequence, KV head) unit.  The query tile is the GQA
-// group times the block width: M = G*K logical rows.  The MMA is always 128 rows high;
-// when M <= 64 (<= 32) the logical rows are replicated 2x (4x) and every replica
-// ("sub-stream") owns a disjoint column range of each key tile, so all 128 softmax
-// threads have work; sub-streams are independent online-softmax streams and are merged
-// at the end exactly like splits.
+// Work decomposition.  A unit is one (sequence, KV head); its query tile is the GQA
+// group times the block width, M = G*K logical rows (row r = i*G + g), padded to the
+// 128 rows of the MMA.  The S CTAs of a thread-block cluster share one unit: each takes
+// an equal share of the unit's 64-position prefix tiles, the last rank also takes the
+// tile of block keys.  Clusters are handed out longest sequence first, so that a ragged
+// batch packs well onto the SMs.
 //
-// Warp roles:
-//   warps 0-3  softmax: thread r owns TMEM lane r: row max, exp2, row sum; bf16
-//              probabilities go to shared memory as the A operand of P.V
-//   warps 4-7  accumulate: thread r keeps output row r (128 fp32) in registers and folds
-//              in each tile's P.V product with the rescale factor of the online softmax
-//   warp 8     producer: barrier set-up and TMA loads of K and V tiles (64-column boxes,
-//              128-byte swizzle) into a ring of stages
-//   warp 9     TMEM allocation and MMA issue (one elected lane)
-// S = Q.K^T is double-buffered in TMEM so QK(t+1) overlaps softmax(t); each P.V product
-// lands in one of two TMEM buffers and is drained by the accumulate warps.
+// One CTA (192 threads, 112 KB of shared memory, 256 TMEM columns: two fit on an SM).
+//   warps 0-3  softmax.  Thread r owns TMEM lane r = query row r: it reads the 64 scores
+//              of a tile, keeps the running max / sum of the online softmax, and writes
+//              the bf16 probabilities back into TMEM over the scores, where the P.V
+//              product reads them as its A operand.
+//   warp 4     producer: one lane issues every TMA load (Q tile, K and V tiles of the
+//              cache, the block K/V tile) into a ring of five 16 KB slots.
+//   warp 5     TMEM allocation and MMA issue: S = Q.K^T into one of two score buffers
+//              (so that QK(t+1) runs under softmax(t)), then O += P.V.
+// The output accumulator O stays in TMEM for the whole CTA.  The running max is only
+// raised when a tile exceeds it by more than 2^8; then, and only then, the owner threads
+// rescale their O rows in TMEM.  Probabilities are bounded by 2^8, which fp32 sums and
+// bf16 operands carry without loss, and the result is the exact softmax because the
+// same shift is used for the numerator and the denominator.
 //
-// The splits of one unit form a thread-block cluster (<= 16 CTAs).  At the end every CTA
-// publishes its partial rows (running max, running sum, unnormalised output) in its own
-// shared memory; after a cluster barrier each CTA merges a slice of the rows straight out
-// of its peers' shared memory (DSMEM) and writes the final bf16 output: no partials in
-// global memory, no second kernel.  More than 16 splits fall back to global partials and
-// the separate merge kernel.
+// Merge.  Every CTA publishes its partial rows (max, sum, unnormalised O) in its own
+// shared memory; after a cluster barrier each CTA merges a slice of the rows straight
+// out of its peers' shared memory and writes the final bf16 rows.  No partial result
+// touches global memory and there is no second kernel.
+//
+// Programmatic dependent launch.  The kernel waits for the preceding kernel of the
+// stream (griddepcontrol.wait) before it reads anything that kernel may have written,
+// and then lets its own successor start.  With ORTHRUS_LAYER_CACHE_QUIESCENT the prefix
+// K/V tiles are requested before that wait, so the next call's loads are in flight
+// while this call is still computing.
 //
 // Every mbarrier wait is bounded: on expiry the CTA records ORTHRUS_DEV_WAIT_TIMEOUT in
 // the status word, drains the copies it armed, still takes part in the cluster barriers,
@@ -35,46 +43,36 @@
 #include "common.cuh"
 
 namespace orthrus {
-#ifdef ORTHRUS_TC_TRACE
-// development aid: per-CTA time stamps (ns) at fixed points, read back by a debug export
-__device__ unsigned long long g_trace[4096 * 32];
-#endif
 namespace {
 
 constexpr int HD = 128;                  // head_dim
 constexpr int MROWS = 128;               // MMA M
-constexpr int NTHREADS = 320;
-constexpr int PSUB_BYTES = 128 * 128;    // a [128 rows][64 cols] bf16 sub-tile (Q, P)
-constexpr int STAGE_BYTES_ALL = 64 * 1024;   // K ring and V ring, each
+constexpr int TN = 64;                   // key positions per tile
+constexpr int NTHREADS = 192;
+constexpr int NSLOT = 5;                 // ring slots, one K or V tile each
+constexpr int QSUB_BYTES = MROWS * 128;  // a [128 rows][64 cols] bf16 sub-tile of Q
+constexpr int SUB_BYTES = TN * 128;      // a [64 rows][64 cols] bf16 sub-tile of K or V
+constexpr int SLOT_BYTES = 2 * SUB_BYTES;
 
 // shared memory map (offsets from a 1024-byte aligned base)
-constexpr int OFF_Q = 0;                               // [128][128] bf16
-constexpr int OFF_P = OFF_Q + 2 * PSUB_BYTES;          // [128][TN] bf16
-constexpr int OFF_K = OFF_P + 2 * PSUB_BYTES;          // K ring; reused for the partial rows
-constexpr int OFF_V = OFF_K + STAGE_BYTES_ALL;         // V ring
-constexpr int OFF_ALPHA = OFF_V + STAGE_BYTES_ALL;     // float [2][128]
-constexpr int OFF_ML = OFF_ALPHA + 2 * 128 * 4;        // float [128][2]
-constexpr int OFF_BAR = OFF_ML + 128 * 2 * 4;          // mbarriers
-constexpr int NUM_BARS = 32;
-constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;       // tmem base, abort flag
+constexpr int OFF_Q = 0;                                   // [128][128] bf16, 2 sub-tiles
+constexpr int OFF_RING = OFF_Q + 2 * QSUB_BYTES;           // NSLOT x 16 KB
+constexpr int OFF_OPART = OFF_RING;                        // float [128][128], after the last MMA
+constexpr int OFF_ML = OFF_OPART + MROWS * HD * 4;         // float [128][2], inside the ring
+constexpr int OFF_BAR = OFF_RING + NSLOT * SLOT_BYTES;     // mbarriers
+constexpr int OFF_MISC = OFF_BAR + 24 * 8;                 // tmem base, abort flag, unit
 constexpr int SMEM_BYTES = OFF_MISC + 64;
-constexpr int OFF_OPART = OFF_K;                       // float [128][128], chunk-swizzled
+static_assert(OFF_ML + MROWS * 8 <= OFF_BAR, "partial rows must fit in the idle ring");
+static_assert(2 * (SMEM_BYTES + 1024) <= 228 * 1024, "two CTAs per SM");
 
-enum { BAR_KFULL = 0, BAR_VFULL = 4, BAR_KEMPTY = 8, BAR_VEMPTY = 12, BAR_SFULL = 16,
-       BAR_OFULL = 18, BAR_OFREE = 20, BAR_AFULL = 22, BAR_PFULL = 24 };
+enum { BAR_FULL = 0, BAR_EMPTY = NSLOT, BAR_QFULL = 2 * NSLOT, BAR_SFULL, BAR_PFULL = BAR_SFULL + 2,
+       BAR_PVDONE = BAR_PFULL + 2, BAR_ALLDONE, NUM_BARS };
+static_assert(NUM_BARS <= 24, "barrier area");
+
+constexpr uint32_t TM_O = 0, TM_S = 128, TM_COLS = 256;   // TMEM column map
+constexpr float RESCALE_THRESHOLD = 8.f;                  // log2 units
 
 __device__ inline uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-#ifdef ORTHRUS_TC_TRACE
-__device__ inline unsigned long long gtimer() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-#define TRACE(slot) do { if ((slot) < 32) g_trace[((blockIdx.y * gridDim.x + blockIdx.x) & 4095) * 32 + (slot)] = gtimer(); } while (0)
-#else
-#define TRACE(slot) do { } while (0)
-#endif
 
 __device__ inline void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
@@ -106,15 +104,31 @@ __device__ inline bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *ab
     *abort_flag = 1;
     return false;
 }
+// the same for a whole warp: every lane learns the common outcome, so that warp-wide
+// (.aligned) instructions behind it are executed by all lanes or by none
+__device__ inline bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+}
 
 __device__ inline void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
                  " [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
+__device__ inline void tma_load_4d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, int c2, int c3,
+                                   uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%2, %3, %4, %5}], [%6];"
+                 ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
+__device__ inline void prefetch_map(const CUtensorMap *tm) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
+}
 __device__ inline void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ inline void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ inline void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ inline void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -154,18 +168,24 @@ __device__ inline uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_
 __host__ __device__ constexpr uint32_t make_idesc(uint32_t n, uint32_t b_mn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
-
-__device__ inline void umma(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+// D[tmem] (+)= A[smem] . B[smem]
+__device__ inline void umma_ss(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
     asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
                  " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
                  ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] . B[smem]   (A: one row per lane, two bf16 per 32-bit column)
+__device__ inline void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                 " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc) : "memory");
 }
 __device__ inline void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
                  ::"r"(bar) : "memory");
 }
-// 32 consecutive fp32 columns of this thread's TMEM lane (no wait: pair with tmem_ld_wait)
-__device__ inline void tmem_ld32_nowait(uint32_t taddr, uint32_t *r) {
+// 32 consecutive 32-bit columns of this thread's TMEM lane (no wait: pair with tmem_ld_wait)
+__device__ inline void tmem_ld32(uint32_t taddr, uint32_t *r) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
                  "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
                  "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
@@ -178,6 +198,18 @@ __device__ inline void tmem_ld32_nowait(uint32_t taddr, uint32_t *r) {
                  : "r"(taddr));
 }
 __device__ inline void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ inline void tmem_st32(uint32_t taddr, const uint32_t *r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+                 "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),
+                   "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]),
+                   "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
+                   "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+                   "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+                 : "memory");
+}
+__device__ inline void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ inline float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -193,390 +225,386 @@ __device__ inline uint32_t sw_off(int r, int c, int sub_bytes) {
     return (uint32_t)((c >> 3) * sub_bytes + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
-template <int TN, int NSUB>
-__global__ void __launch_bounds__(NTHREADS, 1)
-attend_tc_kernel(AttnParams p, const __grid_constant__ CUtensorMap tm_k,
-                 const __grid_constant__ CUtensorMap tm_v, int cluster_size)
-{
-    constexpr int NSTAGE = STAGE_BYTES_ALL / (TN * 256);      // 2 (TN=128) or 4 (TN=64)
-    constexpr int KSUB_BYTES = TN * 128;                      // a [TN][64] bf16 sub-tile
-    constexpr int TILE_BYTES = 2 * KSUB_BYTES;
-    constexpr int W = TN / NSUB;                              // score columns per thread
-    constexpr int MPAD = MROWS / NSUB;                        // logical rows per sub-stream
-    constexpr uint32_t TM_S = 0, TM_O = 2 * TN;               // TMEM column bases
-    static_assert(W % 32 == 0, "a thread reads whole 32-column TMEM chunks");
+struct TcMaps { CUtensorMap k, v, q, kb, vb; };
 
+__global__ void __launch_bounds__(NTHREADS, 2)
+attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const int S, const int kb_rows,
+                 const int quiescent)
+{
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t sbase = smem_u32(smem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + OFF_MISC + 8);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + OFF_MISC);
-    float *alpha_buf = reinterpret_cast<float *>(smem + OFF_ALPHA);
-    float *ml_buf = reinterpret_cast<float *>(smem + OFF_ML);
+    volatile int *seq_slot = reinterpret_cast<volatile int *>(smem + OFF_MISC + 16);
     auto bar = [&](int i) { return sbase + OFF_BAR + i * 8; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int unit = blockIdx.x, split = blockIdx.y, rt = blockIdx.z;
-    if (tid == 0) TRACE(0);
-    const int b = unit / p.Hkv, h = unit % p.Hkv;
-    const int P = clamp_cache_len(p, b);
-    const int ls = last_split(P, p.chunk);
-    const int pos0 = split * p.chunk;
-    const int pos1 = min(P, pos0 + p.chunk);
-    const int n_prefix = (split <= ls && pos1 > pos0) ? (pos1 - pos0 + TN - 1) / TN : 0;
-    const int n_blk = (split == ls) ? 1 : 0;                 // the block tile comes first
-    const int n_tiles = n_prefix + n_blk;
-    const bool active = n_tiles > 0 && (sbase & 1023u) == 0;  // swizzled tiles need 1 KB alignment
-    const int rows_here = min(p.M - rt * MROWS, MPAD);        // logical rows of this row tile
+    const int rank = S > 1 ? (int)cluster_rank() : 0;
+    const int order = blockIdx.y, rt = blockIdx.z;
+    // this row tile: kb_rows block positions x G heads
+    const int i0 = rt * kb_rows;
+    const int rows_here = min(p.K - i0, kb_rows) * p.G;
+    const int n_act = (rows_here + 31) >> 5;                  // softmax warps with rows
+    const bool aligned = (sbase & 1023u) == 0;                // swizzled tiles need 1 KB alignment
 
-    if (tid == 0) *abort_flag = ((sbase & 1023u) != 0) ? 1 : 0;
-
-    const int row_base = (int)((long long)unit * p.capacity);     // row of position 0 in the 2-D maps
-    auto issue_prefix = [&](int t) {                              // t: tile index in this CTA
-        const int st = t % NSTAGE;
-        const int pos = pos0 + (t - n_blk) * TN;
-        const uint32_t kdst = sbase + OFF_K + st * TILE_BYTES;
-        const uint32_t vdst = sbase + OFF_V + st * TILE_BYTES;
-        mbar_expect_tx(bar(BAR_KFULL + st), TILE_BYTES);
-        tma_load_2d(kdst, &tm_k, 0, row_base + pos, bar(BAR_KFULL + st));
-        tma_load_2d(kdst + KSUB_BYTES, &tm_k, 64, row_base + pos, bar(BAR_KFULL + st));
-        mbar_expect_tx(bar(BAR_VFULL + st), TILE_BYTES);
-        tma_load_2d(vdst, &tm_v, 0, row_base + pos, bar(BAR_VFULL + st));
-        tma_load_2d(vdst + KSUB_BYTES, &tm_v, 64, row_base + pos, bar(BAR_VFULL + st));
-    };
-    int produced = n_blk;                    // tiles armed so far (the block tile is armed by the prologue)
-
-    if (active) {
-        if (warp == 8) {
-            if (lane == 0) {
-                for (int i = 0; i < 16; ++i) mbar_init(bar(i), 1);                // k/v full/empty
-                mbar_init(bar(BAR_SFULL), 1); mbar_init(bar(BAR_SFULL + 1), 1);
-                mbar_init(bar(BAR_OFULL), 1); mbar_init(bar(BAR_OFULL + 1), 1);
-                mbar_init(bar(BAR_OFREE), 128); mbar_init(bar(BAR_OFREE + 1), 128);
-                mbar_init(bar(BAR_AFULL), 128); mbar_init(bar(BAR_AFULL + 1), 128);
-                mbar_init(bar(BAR_PFULL), 128);
-                asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-                fence_proxy_async();
-                // the first prefix tiles are requested before anything else happens
-                while (produced < n_tiles && produced < NSTAGE) { issue_prefix(produced); ++produced; }
-            }
-        } else if (warp == 9) {
-            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;"
-                         ::"r"(smem_u32(tmem_slot)) : "memory");
-            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-        } else {
-            // warps 0-7: Q rows (replicated per sub-stream, zero-padded) and, in the owning
-            // split, the block K/V rows (zero-padded to the tile) into the swizzled operand
-            // layout; all global loads are issued before the first store
-            const int t8 = tid;                                   // 0..255
-            const uint4 zero = make_uint4(0, 0, 0, 0);
-            const __nv_bfloat16 *q = static_cast<const __nv_bfloat16 *>(p.q);
-            uint4 qv[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const int e = t8 + k * 256, r = e >> 4, c = e & 15;
-                const int Rl = r % MPAD, R = rt * MROWS + Rl;
-                qv[k] = zero;
-                if (Rl < rows_here) {
-                    const int i = R / p.G, g = R % p.G;
-                    qv[k] = __ldg(reinterpret_cast<const uint4 *>(
-                                q + (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD) + c);
-                }
-            }
-            uint4 kv[4], vv[4];
-            if (n_blk) {
-                const __nv_bfloat16 *kb = static_cast<const __nv_bfloat16 *>(p.k_blk);
-                const __nv_bfloat16 *vb = static_cast<const __nv_bfloat16 *>(p.v_blk);
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {                     // K <= 64 rows x 16 chunks
-                    const int e = t8 + k * 256, r = e >> 4, c = e & 15;
-                    kv[k] = zero; vv[k] = zero;
-                    if (r < p.K) {
-                        const long long off = (((long long)b * p.K + r) * p.Hkv + h) * HD;
-                        kv[k] = __ldg(reinterpret_cast<const uint4 *>(kb + off) + c);
-                        vv[k] = __ldg(reinterpret_cast<const uint4 *>(vb + off) + c);
-                    }
-                }
-            }
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const int e = t8 + k * 256, r = e >> 4, c = e & 15;
-                *reinterpret_cast<uint4 *>(smem + OFF_Q + sw_off(r, c, PSUB_BYTES)) = qv[k];
-            }
-            if (NSUB > 1) {        // columns a sub-stream never writes must read as zero
-                for (int e = t8; e < MROWS * (TN / 8); e += 256)
-                    *reinterpret_cast<uint4 *>(smem + OFF_P + e * 16) = zero;
-            }
-            if (n_blk) {
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int e = t8 + k * 256, r = e >> 4, c = e & 15;
-                    *reinterpret_cast<uint4 *>(smem + OFF_K + sw_off(r, c, KSUB_BYTES)) = kv[k];
-                    *reinterpret_cast<uint4 *>(smem + OFF_V + sw_off(r, c, KSUB_BYTES)) = vv[k];
-                }
-                for (int e = t8 + 1024; e < TN * 16; e += 256) {  // V rows 64..TN-1 of the block tile
-                    const int r = e >> 4, c = e & 15;
-                    *reinterpret_cast<uint4 *>(smem + OFF_V + sw_off(r, c, KSUB_BYTES)) = zero;
-                }
-            }
-            fence_proxy_async();
-        }
-    } else if (tid < MROWS) {
-        ml_buf[tid * 2] = -INFINITY;          // an empty split publishes empty partial rows
-        ml_buf[tid * 2 + 1] = 0.f;
+    // ------------------------------------------------------------------ prologue
+    if (tid == 0) { *abort_flag = aligned ? 0 : 1; *seq_slot = 0; }
+    if (warp == 4 && lane == 0) {
+        for (int i = 0; i < 2 * NSLOT; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(BAR_QFULL), 1);
+        mbar_init(bar(BAR_SFULL), 1); mbar_init(bar(BAR_SFULL + 1), 1);
+        mbar_init(bar(BAR_PFULL), n_act); mbar_init(bar(BAR_PFULL + 1), n_act);
+        mbar_init(bar(BAR_PVDONE), 1);
+        mbar_init(bar(BAR_ALLDONE), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+        prefetch_map(&tm.k); prefetch_map(&tm.v); prefetch_map(&tm.q);
+        prefetch_map(&tm.kb); prefetch_map(&tm.vb);
+    } else if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(TM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = active ? *tmem_slot : 0u;
-    if (tid == 0) TRACE(1);
+    const uint32_t tmem = *tmem_slot;
 
-    if (active && warp < 4) {
+    // Nothing written by earlier work of the stream has been read so far.
+    if (!quiescent) griddep_wait();
+
+    // ------------------------------------------------------------------ which unit
+    // clusters are ordered longest prefix first (ties by sequence index)
+    int b = order / p.Hkv;
+    const int h = order % p.Hkv;
+    const long long len_hi = p.capacity - p.K;
+    if (p.B > 1 && p.B <= 128) {
+        const int want = b;
+        for (int i = tid; i < p.B; i += NTHREADS) {
+            const long long Pi = min(max((long long)__ldg(p.cache_len + i), 0ll), len_hi);
+            int before = 0;
+            for (int j = 0; j < p.B; ++j) {
+                const long long Pj = min(max((long long)__ldg(p.cache_len + j), 0ll), len_hi);
+                before += (Pj > Pi) || (Pj == Pi && j < i);
+            }
+            if (before == want) *seq_slot = i;
+        }
+        __syncthreads();
+        b = *seq_slot;
+    }
+    int P = p.cache_len[b];
+    if (P < 0 || P > len_hi) {
+        if (tid == 0 && rank == 0 && p.status) atomicOr(p.status, ORTHRUS_DEV_BAD_CACHE_LEN);
+        P = P < 0 ? 0 : (int)len_hi;
+    }
+    const int n_pre = (P + TN - 1) / TN;                      // prefix tiles of the unit
+    const int t0 = (int)((long long)rank * n_pre / S);
+    const int t1 = (int)((long long)(rank + 1) * n_pre / S);
+    const int n_mine = t1 - t0;                               // prefix tiles of this CTA
+    const bool owner = rank == S - 1;                         // also takes the block tile, last
+    const int n_tiles = n_mine + (owner ? 1 : 0);
+    const bool active = n_tiles > 0 && aligned;
+    const int row_base = (int)(((long long)b * p.Hkv + h) * p.capacity);   // row of position 0
+
+    // ring item j: tile j/2, K (even) or V (odd); slot j % NSLOT
+    auto issue_item = [&](int j) {
+        const int t = j >> 1, slot = j % NSLOT;
+        const bool is_v = j & 1;
+        const uint32_t dst = sbase + OFF_RING + slot * SLOT_BYTES;
+        const uint32_t fb = bar(BAR_FULL + slot);
+        mbar_expect_tx(fb, SLOT_BYTES);
+        if (t < n_mine) {
+            const CUtensorMap *m = is_v ? &tm.v : &tm.k;
+            const int row = row_base + (t0 + t) * TN;
+            tma_load_2d(dst, m, 0, row, fb);
+            tma_load_2d(dst + SUB_BYTES, m, 64, row, fb);
+        } else {                  // block tile: rows >= K are out of bounds and arrive as zeros
+            const CUtensorMap *m = is_v ? &tm.vb : &tm.kb;
+            tma_load_4d(dst, m, 0, h, 0, b, fb);
+            tma_load_4d(dst + SUB_BYTES, m, 64, h, 0, b, fb);
+        }
+    };
+    int produced = 0;                                         // ring items armed so far
+    if (quiescent) {
+        // the cache rows below cache_len are not being written by the preceding kernel:
+        // request the first prefix tiles before waiting for it
+        if (active && warp == 4 && lane == 0)
+            while (produced < 2 * n_mine && produced < NSLOT) { issue_item(produced); ++produced; }
+        griddep_wait();
+    }
+    griddep_launch();
+
+    if (active && warp < n_act) {
         // ------------------------------------------------------------------ softmax
         const int r = tid;
-        const int sub = r / MPAD, Rl = r % MPAD;
-        const int i_row = (rt * MROWS + Rl) / p.G;
-        const int col0 = sub * W;
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16) + TM_S + col0;
+        const bool valid = r < rows_here;
+        const int i_row = i0 + r / p.G;
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        const float sc = p.scale_log2;
         float m_run = -INFINITY, l_run = 0.f;
-        for (int t = 0; t < n_tiles; ++t) {
-            const int sb = t & 1;
-            if (!mbar_wait(bar(BAR_SFULL + sb), (t >> 1) & 1, abort_flag)) break;
-            tc_fence_after();
-            if (tid == 0) TRACE(4 + 4 * t);
-            uint32_t s[W];
-#pragma unroll
-            for (int c = 0; c < W / 32; ++c) tmem_ld32_nowait(lane_addr + sb * TN + c * 32, s + c * 32);
-            tmem_ld_wait();
-            const bool is_blk = t < n_blk;
-            const int nv = is_blk ? p.K : min(TN, pos1 - (pos0 + (t - n_blk) * TN));
-            // number of visible columns of this thread's range [col0, col0 + W)
-            const int lim = min(W, max(0, ((is_blk && p.causal) ? min(nv, i_row + 1) : nv) - col0));
-            float mx = -INFINITY;
-            if (lim == W) {
-#pragma unroll
-                for (int j = 0; j < W; ++j) mx = fmaxf(mx, __uint_as_float(s[j]));
-            } else {
-#pragma unroll
-                for (int j = 0; j < W; ++j) if (j < lim) mx = fmaxf(mx, __uint_as_float(s[j]));
-            }
-            const float m_new = fmaxf(m_run, mx * p.scale_log2);
-            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;     // nothing visible so far
-            const float alpha = ex2(m_run - m_use);
-            m_run = m_new;
-            if (tid == 0) TRACE(5 + 4 * t);
-            // alpha slot (t&1) was last read by accumulate(t-2); P was last read by PV(t-1)
-            if (t >= 2 && !mbar_wait(bar(BAR_OFREE + sb), ((t - 2) >> 1) & 1, abort_flag)) break;
-            alpha_buf[sb * 128 + r] = alpha;
-            mbar_arrive(bar(BAR_AFULL + sb));
-            if (t >= 1 && !mbar_wait(bar(BAR_OFULL + ((t - 1) & 1)), ((t - 1) >> 1) & 1, abort_flag)) break;
-            float lsum = 0.f;
-#pragma unroll
-            for (int c8 = 0; c8 < W / 8; ++c8) {
-                uint32_t w[4];
-#pragma unroll
-                for (int j = 0; j < 8; j += 2) {
-                    const int col = c8 * 8 + j;
-                    float p0 = ex2(fmaf(__uint_as_float(s[col]), p.scale_log2, -m_use));
-                    float p1 = ex2(fmaf(__uint_as_float(s[col + 1]), p.scale_log2, -m_use));
-                    if (lim != W) {
-                        if (col >= lim) p0 = 0.f;
-                        if (col + 1 >= lim) p1 = 0.f;
-                    }
-                    lsum += p0 + p1;
-                    w[j >> 1] = pack_bf16(p0, p1);
-                }
-                *reinterpret_cast<uint4 *>(smem + OFF_P + sw_off(r, col0 / 8 + c8, PSUB_BYTES)) =
-                    make_uint4(w[0], w[1], w[2], w[3]);
-            }
-            l_run = l_run * alpha + lsum;
-            fence_proxy_async();
-            tc_fence_before();
-            mbar_arrive(bar(BAR_PFULL));
-            if (tid == 0) TRACE(6 + 4 * t);
-        }
-        ml_buf[r * 2] = m_run;
-        ml_buf[r * 2 + 1] = l_run;
-    } else if (active && warp < 8) {
-        // ------------------------------------------------------------------ accumulate
-        const int r = tid - 128;
-        const uint32_t lane_addr = tmem + ((uint32_t)((warp - 4) * 32) << 16) + TM_O;
-        float o[HD];
-#pragma unroll
-        for (int j = 0; j < HD; ++j) o[j] = 0.f;
         bool ok = true;
         for (int t = 0; t < n_tiles; ++t) {
-            const int ob = t & 1;
-            if (!mbar_wait(bar(BAR_AFULL + ob), (t >> 1) & 1, abort_flag)) { ok = false; break; }
-            const float alpha = alpha_buf[ob * 128 + r];
-            if (!mbar_wait(bar(BAR_OFULL + ob), (t >> 1) & 1, abort_flag)) { ok = false; break; }
+            const int sb = t & 1;
+            ok = mbar_wait_warp(bar(BAR_SFULL + sb), (t >> 1) & 1, abort_flag);
+            if (!ok) break;
             tc_fence_after();
+            uint32_t s[TN];
+            tmem_ld32(lane_base + TM_S + sb * TN, s);
+            tmem_ld32(lane_base + TM_S + sb * TN + 32, s + 32);
+            tmem_ld_wait();
+            // visible columns of this row in this tile
+            int lim;
+            if (t < n_mine) lim = min(TN, P - (t0 + t) * TN);
+            else lim = p.causal ? min(p.K, i_row + 1) : p.K;
+            if (!valid) lim = 0;
+            float mx = -INFINITY;
+            if (lim == TN) {
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                uint32_t v[32];
-                tmem_ld32_nowait(lane_addr + ob * 128 + c4 * 32, v);
-                tmem_ld_wait();
+                for (int j = 0; j < TN; ++j) mx = fmaxf(mx, __uint_as_float(s[j]));
+            } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    o[c4 * 32 + j] = fmaf(o[c4 * 32 + j], alpha, __uint_as_float(v[j]));
+                for (int j = 0; j < TN; ++j) if (j < lim) mx = fmaxf(mx, __uint_as_float(s[j]));
             }
-            tc_fence_before();
-            mbar_arrive(bar(BAR_OFREE + ob));
-            if (tid == 128) TRACE(7 + 4 * t);
-        }
-        // publish the partial row; the K ring is idle once the last P.V product has landed
-        if (ok) {
+            const float m_new = fmaxf(m_run, mx * sc);
+            const bool need = m_new > m_run + RESCALE_THRESHOLD;   // also the first finite maximum
+            if (__any_sync(0xffffffffu, need)) {
+                const float alpha = need ? ex2(m_run - m_new) : 1.f;
+                if (need) { m_run = m_new; l_run *= alpha; }
+                if (t > 0) {
+                    // O holds the products of tiles 0..t-1 and nothing is adding to it now
+                    ok = mbar_wait_warp(bar(BAR_PVDONE), (t - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c4 = 0; c4 < HD / 32; ++c4) {
+                        uint32_t o[32];
+                        tmem_ld32(lane_base + TM_O + c4 * 32, o);
+                        tmem_ld_wait();
 #pragma unroll
-            for (int c = 0; c < 32; ++c)
-                *reinterpret_cast<float4 *>(smem + OFF_OPART + r * 512 + ((c ^ (r & 31)) << 4)) =
-                    make_float4(o[c * 4], o[c * 4 + 1], o[c * 4 + 2], o[c * 4 + 3]);
+                        for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+                        tmem_st32(lane_base + TM_O + c4 * 32, o);
+                    }
+                }
+            }
+            const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
+            uint32_t pk[TN / 2];
+            float lsum = 0.f;
+            if (lim == TN) {
+#pragma unroll
+                for (int j = 0; j < TN; j += 2) {
+                    const float p0 = ex2(fmaf(__uint_as_float(s[j]), sc, neg_m));
+                    const float p1 = ex2(fmaf(__uint_as_float(s[j + 1]), sc, neg_m));
+                    lsum += p0 + p1;
+                    pk[j >> 1] = pack_bf16(p0, p1);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < TN; j += 2) {
+                    float p0 = ex2(fmaf(__uint_as_float(s[j]), sc, neg_m));
+                    float p1 = ex2(fmaf(__uint_as_float(s[j + 1]), sc, neg_m));
+                    if (j >= lim) p0 = 0.f;
+                    if (j + 1 >= lim) p1 = 0.f;
+                    lsum += p0 + p1;
+                    pk[j >> 1] = pack_bf16(p0, p1);
+                }
+            }
+            l_run += lsum;
+            tmem_st32(lane_base + TM_S + sb * TN, pk);         // P over the scores, 2 bf16 per column
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_PFULL + sb));
         }
-    } else if (active && warp == 8) {
+        // BAR_PVDONE cannot be used here: a parity wait cannot tell phase k from phase k-2, and
+        // by now the barrier may be one or two phases ahead of what this thread last observed
+        if (ok) ok = mbar_wait_warp(bar(BAR_ALLDONE), 0, abort_flag);
+        if (ok) {
+            tc_fence_after();
+            if (S == 1) {
+                // the whole unit was here: normalise and write the final rows
+                const float inv = 1.f / l_run;
+                __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.out) +
+                    (((long long)b * p.K + i_row) * p.Hq + h * p.G + (r % p.G)) * HD;
+#pragma unroll 1
+                for (int c4 = 0; c4 < HD / 32; ++c4) {
+                    uint32_t o[32];
+                    tmem_ld32(lane_base + TM_O + c4 * 32, o);
+                    tmem_ld_wait();
+                    if (valid) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint4 w;
+                            w.x = pack_bf16(__uint_as_float(o[c * 8 + 0]) * inv, __uint_as_float(o[c * 8 + 1]) * inv);
+                            w.y = pack_bf16(__uint_as_float(o[c * 8 + 2]) * inv, __uint_as_float(o[c * 8 + 3]) * inv);
+                            w.z = pack_bf16(__uint_as_float(o[c * 8 + 4]) * inv, __uint_as_float(o[c * 8 + 5]) * inv);
+                            w.w = pack_bf16(__uint_as_float(o[c * 8 + 6]) * inv, __uint_as_float(o[c * 8 + 7]) * inv);
+                            reinterpret_cast<uint4 *>(dst)[c4 * 4 + c] = w;
+                        }
+                    }
+                }
+            } else {
+                // publish the partial row; the ring is idle once the last product has landed
+#pragma unroll 1
+                for (int c4 = 0; c4 < HD / 32; ++c4) {
+                    uint32_t o[32];
+                    tmem_ld32(lane_base + TM_O + c4 * 32, o);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        *reinterpret_cast<uint4 *>(smem + OFF_OPART + r * 512 + (((c4 * 8 + c) ^ (r & 31)) << 4)) =
+                            make_uint4(o[c * 4], o[c * 4 + 1], o[c * 4 + 2], o[c * 4 + 3]);
+                }
+                float *ml = reinterpret_cast<float *>(smem + OFF_ML);
+                ml[r * 2] = m_run;
+                ml[r * 2 + 1] = l_run;
+            }
+        }
+        tc_fence_before();
+    } else if (active && warp == 4) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            if (n_blk) { mbar_arrive(bar(BAR_KFULL)); mbar_arrive(bar(BAR_VFULL)); }
+            // the query rows of this tile: box = 64 columns x G heads x kb_rows positions
+            mbar_expect_tx(bar(BAR_QFULL), (uint32_t)(2 * 128 * p.G * kb_rows));
+            tma_load_4d(sbase + OFF_Q, &tm.q, 0, h * p.G, i0, b, bar(BAR_QFULL));
+            tma_load_4d(sbase + OFF_Q + QSUB_BYTES, &tm.q, 64, h * p.G, i0, b, bar(BAR_QFULL));
             bool ok = true;
-            for (int t = produced; t < n_tiles && ok; ++t) {
-                const int st = t % NSTAGE, use = t / NSTAGE;
-                // the stage was last used by tile t-NSTAGE: K is free after its QK, V after its PV
-                ok = mbar_wait(bar(BAR_KEMPTY + st), (use - 1) & 1, abort_flag) &&
-                     mbar_wait(bar(BAR_VEMPTY + st), (use - 1) & 1, abort_flag);
-                if (ok) { issue_prefix(t); produced = t + 1; }
+            const int n_items = 2 * n_tiles;
+            while (produced < n_items && ok) {
+                const int slot = produced % NSLOT, use = produced / NSLOT;
+                if (use > 0) ok = mbar_wait(bar(BAR_EMPTY + slot), (use - 1) & 1, abort_flag);
+                if (ok) { issue_item(produced); ++produced; }
             }
             if (*abort_flag) {
                 // give the copies that were armed a bounded time to land before smem is released
-                for (int t = n_blk; t < produced; ++t) {
+                for (int j = max(0, produced - NSLOT); j < produced; ++j) {   // latest use of each slot
                     int dummy = 0;
-                    mbar_wait(bar(BAR_KFULL + t % NSTAGE), (t / NSTAGE) & 1, &dummy);
-                    dummy = 0;
-                    mbar_wait(bar(BAR_VFULL + t % NSTAGE), (t / NSTAGE) & 1, &dummy);
+                    mbar_wait(bar(BAR_FULL + j % NSLOT), (j / NSLOT) & 1, &dummy);
                 }
+                int dummy = 0;
+                mbar_wait(bar(BAR_QFULL), 0, &dummy);
             }
         }
-    } else if (active) {
+    } else if (active && warp == 5) {
         // ------------------------------------------------------------------ MMA issue
-        const uint32_t q_addr = sbase + OFF_Q, p_addr = sbase + OFF_P;
+        const uint32_t q_addr = sbase + OFF_Q;
         constexpr uint32_t IDESC_QK = make_idesc(TN, 0);      // A = Q, B = K tile, both K-major
-        constexpr uint32_t IDESC_PV = make_idesc(HD, 1);      // A = P (K-major), B = V tile (MN-major)
+        constexpr uint32_t IDESC_PV = make_idesc(HD, 1);      // A = P (TMEM), B = V tile (MN-major)
         auto issue_qk = [&](int t) -> bool {
-            const int st = t % NSTAGE;
-            if (!mbar_wait(bar(BAR_KFULL + st), (t / NSTAGE) & 1, abort_flag)) return false;
+            const int j = 2 * t, slot = j % NSLOT;
+            if (!mbar_wait_warp(bar(BAR_FULL + slot), (j / NSLOT) & 1, abort_flag)) return false;
             tc_fence_after();
             if (lane == 0) {
-                if (t < 4) TRACE(24 + t);
-                const uint32_t k_addr = sbase + OFF_K + st * TILE_BYTES;
+                const uint32_t k_addr = sbase + OFF_RING + slot * SLOT_BYTES;
 #pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {       // 16 head-dim columns per MMA
-                    umma(tmem + TM_S + (t & 1) * TN,
-                         make_desc(q_addr + (kk >> 2) * PSUB_BYTES + (kk & 3) * 32, 16, 1024),
-                         make_desc(k_addr + (kk >> 2) * KSUB_BYTES + (kk & 3) * 32, 16, 1024),
-                         IDESC_QK, kk > 0);
+                for (int kk = 0; kk < HD / 16; ++kk) {        // 16 head-dim columns per MMA
+                    umma_ss(tmem + TM_S + (t & 1) * TN,
+                            make_desc(q_addr + (kk >> 2) * QSUB_BYTES + (kk & 3) * 32, 16, 1024),
+                            make_desc(k_addr + (kk >> 2) * SUB_BYTES + (kk & 3) * 32, 16, 1024),
+                            IDESC_QK, kk > 0);
                 }
-                umma_commit(bar(BAR_KEMPTY + st));
+                umma_commit(bar(BAR_EMPTY + slot));
                 umma_commit(bar(BAR_SFULL + (t & 1)));
             }
             __syncwarp();
             return true;
         };
-        auto issue_pv = [&](int u) -> bool {
-            const int st = u % NSTAGE;
-            if (!mbar_wait(bar(BAR_VFULL + st), (u / NSTAGE) & 1, abort_flag)) return false;
-            // a ragged prefix tile: V rows past the chunk end may hold anything, and 0 * NaN
-            // would poison the product, so they are cleared before the MMA reads them
-            const bool is_blk = u < n_blk;
-            const int nv = is_blk ? TN : min(TN, pos1 - (pos0 + (u - n_blk) * TN));
+        auto issue_pv = [&](int t) -> bool {
+            const int j = 2 * t + 1, slot = j % NSLOT;
+            if (!mbar_wait_warp(bar(BAR_FULL + slot), (j / NSLOT) & 1, abort_flag)) return false;
+            // a ragged prefix tile: V rows past the prefix may hold anything, and 0 * NaN would
+            // poison the product, so they are cleared before the MMA reads them
+            const int nv = t < n_mine ? min(TN, P - (t0 + t) * TN) : TN;
             if (nv < TN) {
-                unsigned char *vt = smem + OFF_V + st * TILE_BYTES;
+                unsigned char *vt = smem + OFF_RING + slot * SLOT_BYTES;
                 for (int e = lane; e < (TN - nv) * 16; e += 32) {
                     const int rr = nv + (e >> 4), c = e & 15;
-                    *reinterpret_cast<uint4 *>(vt + sw_off(rr, c, KSUB_BYTES)) = make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4 *>(vt + sw_off(rr, c, SUB_BYTES)) = make_uint4(0, 0, 0, 0);
                 }
                 fence_proxy_async();
                 __syncwarp();
             }
-            if (!mbar_wait(bar(BAR_PFULL), u & 1, abort_flag)) return false;
-            if (u >= 2 && !mbar_wait(bar(BAR_OFREE + (u & 1)), ((u - 2) >> 1) & 1, abort_flag)) return false;
+            if (!mbar_wait_warp(bar(BAR_PFULL + (t & 1)), (t >> 1) & 1, abort_flag)) return false;
             tc_fence_after();
             if (lane == 0) {
-                const uint32_t v_addr = sbase + OFF_V + st * TILE_BYTES;
+                const uint32_t v_addr = sbase + OFF_RING + slot * SLOT_BYTES;
 #pragma unroll
-                for (int kk = 0; kk < TN / 16; ++kk) {       // 16 key positions per MMA
-                    umma(tmem + TM_O + (u & 1) * 128,
-                         make_desc(p_addr + (kk >> 2) * PSUB_BYTES + (kk & 3) * 32, 16, 1024),
-                         make_desc(v_addr + kk * 2048, KSUB_BYTES, 1024), IDESC_PV, kk > 0);
+                for (int kk = 0; kk < TN / 16; ++kk) {        // 16 key positions per MMA
+                    umma_ts(tmem + TM_O, tmem + TM_S + (t & 1) * TN + kk * 8,
+                            make_desc(v_addr + kk * 2048, SUB_BYTES, 1024), IDESC_PV, (t > 0) || (kk > 0));
                 }
-                umma_commit(bar(BAR_VEMPTY + st));
-                umma_commit(bar(BAR_OFULL + (u & 1)));
+                umma_commit(bar(BAR_EMPTY + slot));
+                umma_commit(bar(BAR_PVDONE));
+                if (t == n_tiles - 1) umma_commit(bar(BAR_ALLDONE));
             }
             __syncwarp();
             return true;
         };
-        bool ok = true;
+        bool ok = mbar_wait_warp(bar(BAR_QFULL), 0, abort_flag);
+        if (ok) { tc_fence_after(); ok = issue_qk(0); }
         for (int t = 0; t < n_tiles && ok; ++t) {
-            ok = issue_qk(t);
-            if (ok && t > 0) ok = issue_pv(t - 1);
+            if (t + 1 < n_tiles) ok = issue_qk(t + 1);
+            if (ok) ok = issue_pv(t);
         }
-        if (ok) ok = issue_pv(n_tiles - 1);
-        if (ok)    // every MMA must have retired before the K ring is reused and TMEM is freed
-            mbar_wait(bar(BAR_OFULL + ((n_tiles - 1) & 1)), ((n_tiles - 1) >> 1) & 1, abort_flag);
+        // every MMA must have retired before the ring is reused and TMEM is freed
+        if (ok) mbar_wait_warp(bar(BAR_ALLDONE), 0, abort_flag);
+        tc_fence_before();
+    } else if (!active && S > 1 && tid < MROWS) {
+        float *ml = reinterpret_cast<float *>(smem + OFF_ML);
+        ml[tid * 2] = -INFINITY;              // a CTA without tiles publishes empty partial rows
+        ml[tid * 2 + 1] = 0.f;
     }
 
     // ---------------------------------------------------------------------- merge
-    tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (tid == 0) TRACE(2);
-    if (active && warp == 9)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+    if (warp == 5)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TM_COLS) : "memory");
     if (tid == 0 && *abort_flag && p.status) atomicOr(p.status, ORTHRUS_DEV_WAIT_TIMEOUT);
-    if (cluster_size > 1) cluster_sync_all();
+    if (S == 1) return;
+    cluster_sync_all();
 
-    const int my_rank = cluster_size > 1 ? (int)cluster_rank() : 0;
-    const int n_part = cluster_size * NSUB;                   // <= 32 partial rows per logical row
-    const bool final_out = (cluster_size == p.n_splits);
-    if (warp < 8) {
-        const int pj_rank = lane / NSUB, pj_sub = lane % NSUB;
-        for (int Rl = my_rank + cluster_size * warp; Rl < rows_here; Rl += cluster_size * 8) {
-            float mj = -INFINITY, lj = 0.f;
-            if (lane < n_part) {
-                const uint32_t a = sbase + OFF_ML + (pj_sub * MPAD + Rl) * 8;
-                const float2 v = ld_cluster_f2(cluster_size > 1 ? map_to_rank(a, pj_rank) : a);
-                mj = v.x; lj = v.y;
+    // rank k merges rows k, k+S, ...: lane j holds the weight of partial j, every lane four
+    // output columns
+    for (int Rl = rank + S * warp; Rl < rows_here; Rl += S * (NTHREADS / 32)) {
+        float mj = -INFINITY, lj = 0.f;
+        if (lane < S) {
+            const float2 v = ld_cluster_f2(map_to_rank(sbase + OFF_ML + Rl * 8, lane));
+            mj = v.x; lj = v.y;
+        }
+        float mmax = mj;
+#pragma unroll
+        for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
+        const float wj = (lj > 0.f) ? ex2(mj - mmax) : 0.f;
+        float L = wj * lj;
+#pragma unroll
+        for (int off = 16; off; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
+        const uint32_t local = sbase + OFF_OPART + Rl * 512 + ((lane ^ (Rl & 31)) << 4);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int j0 = 0; j0 < S; j0 += 8) {
+            float4 v[8];
+            float w[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int j = min(j0 + u, S - 1);
+                w[u] = (j0 + u < S) ? __shfl_sync(0xffffffffu, wj, j) : 0.f;
+                v[u] = ld_cluster_f4(map_to_rank(local, j));
             }
-            float mmax = mj;
 #pragma unroll
-            for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
-            const float wj = (lj > 0.f) ? ex2(mj - mmax) : 0.f;
-            float L = wj * lj;
-#pragma unroll
-            for (int off = 16; off; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-            for (int j = 0; j < n_part; ++j) {
-                const float w = __shfl_sync(0xffffffffu, wj, j);
-                if (w != 0.f) {
-                    const int row = (j % NSUB) * MPAD + Rl;
-                    const uint32_t a = sbase + OFF_OPART + row * 512 + ((lane ^ (row & 31)) << 4);
-                    const float4 v = ld_cluster_f4(cluster_size > 1 ? map_to_rank(a, j / NSUB) : a);
-                    acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y);
-                    acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+            for (int u = 0; u < 8; ++u) {
+                // an empty partial has weight 0 and unwritten rows: keep them out of the sum
+                if (w[u] != 0.f) {
+                    acc.x = fmaf(w[u], v[u].x, acc.x); acc.y = fmaf(w[u], v[u].y, acc.y);
+                    acc.z = fmaf(w[u], v[u].z, acc.z); acc.w = fmaf(w[u], v[u].w, acc.w);
                 }
             }
-            const int R = rt * MROWS + Rl;
-            if (final_out) {
-                const int i = R / p.G, g = R % p.G;
-                const float inv = 1.f / L;
-                uint2 *dst = reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) +
-                             (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD);
-                dst[lane] = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
-            } else {
-                const long long row = ((long long)unit * p.n_splits + split) * p.M + R;
-                reinterpret_cast<float4 *>(p.part_o + row * HD)[lane] = acc;
-                if (lane == 0) { p.part_ml[row * 2] = mmax; p.part_ml[row * 2 + 1] = L; }
-            }
         }
+        const int i = i0 + Rl / p.G, g = Rl % p.G;
+        const float inv = 1.f / L;
+        uint2 *dst = reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) +
+                     (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD);
+        dst[lane] = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
     }
-    if (cluster_size > 1) cluster_sync_all();     // peers may still be reading this CTA's rows
-    if (tid == 0) TRACE(3);
+    cluster_sync_all();     // peers may still be reading this CTA's rows
 }
 
 // ---------------------------------------------------------------------------- host side
@@ -600,35 +628,43 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-// 2-D view of a cache tensor: rows = B*Hkv*capacity positions, 128 bf16 columns;
-// box = 64 columns x `box_rows` rows, 128-byte swizzle.  Maps are cached by key.
+// Tensor maps over bf16 tensors whose innermost dimension is the 128-wide head: up to four
+// dimensions, boxes of 64 columns with the 128-byte swizzle.  Cached by (pointer, shape).
 struct MapKey {
-    const void *ptr; unsigned long long rows; int box_rows;
-    bool operator==(const MapKey &o) const { return ptr == o.ptr && rows == o.rows && box_rows == o.box_rows; }
+    const void *ptr; unsigned long long d1, d2, d3; unsigned b1, b2;
+    bool operator==(const MapKey &o) const {
+        return ptr == o.ptr && d1 == o.d1 && d2 == o.d2 && d3 == o.d3 && b1 == o.b1 && b2 == o.b2;
+    }
 };
 struct MapKeyHash {
     size_t operator()(const MapKey &k) const {
-        return std::hash<const void *>()(k.ptr) ^ (std::hash<unsigned long long>()(k.rows) * 0x9E3779B97F4A7C15ull) ^
-               (size_t)k.box_rows;
+        size_t x = std::hash<const void *>()(k.ptr);
+        for (unsigned long long v : {k.d1, k.d2, k.d3, (unsigned long long)k.b1, (unsigned long long)k.b2})
+            x = (x ^ v) * 0x9E3779B97F4A7C15ull;
+        return x;
     }
 };
 
-bool get_map(const void *ptr, unsigned long long rows, int box_rows, CUtensorMap *out)
+// dims: (128, d1, d2, d3) row-major with d3 outermost; box (64, b1, b2, 1).  rank = 2 when
+// d2 == 0 (then the box is (64, b1)).
+bool get_map(const void *ptr, unsigned long long d1, unsigned long long d2, unsigned long long d3,
+             unsigned b1, unsigned b2, CUtensorMap *out)
 {
     static std::mutex mu;
     static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
     std::lock_guard<std::mutex> lock(mu);
-    const MapKey key{ptr, rows, box_rows};
+    const MapKey key{ptr, d1, d2, d3, b1, b2};
     auto it = cache.find(key);
     if (it != cache.end()) { *out = it->second; return true; }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)HD, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)HD * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-    const cuuint32_t estr[2] = {1, 1};
+    const int rank = d2 == 0 ? 2 : 4;
+    const cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)d1, (cuuint64_t)d2, (cuuint64_t)d3};
+    const cuuint64_t strides[3] = {(cuuint64_t)HD * 2, (cuuint64_t)HD * 2 * d1, (cuuint64_t)HD * 2 * d1 * d2};
+    const cuuint32_t box[4] = {64, b1, b2, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
     CUtensorMap tm;
-    const CUresult r = fn(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims,
+    const CUresult r = fn(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(ptr), dims,
                           strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -639,73 +675,70 @@ bool get_map(const void *ptr, unsigned long long rows, int box_rows, CUtensorMap
     return true;
 }
 
-template <int TN, int NSUB>
-cudaError_t launch_one(const AttnParams &p, int cluster, cudaStream_t st)
-{
-    const unsigned long long rows = (unsigned long long)p.B * p.Hkv * p.capacity;
-    CUtensorMap tk, tv;
-    if (!get_map(p.k_cache, rows, TN, &tk) || !get_map(p.v_cache, rows, TN, &tv)) return cudaErrorInvalidValue;
-    auto kern = attend_tc_kernel<TN, NSUB>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.B * p.Hkv, p.n_splits, (p.M + MROWS - 1) / MROWS);
-    cfg.blockDim = dim3(NTHREADS);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    int n_attr = 0;
-    if (cluster > 1) {
-        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
-        attr[n_attr].val.clusterDim.x = 1;
-        attr[n_attr].val.clusterDim.y = cluster;
-        attr[n_attr].val.clusterDim.z = 1;
-        ++n_attr;
-    }
-    cfg.attrs = attr;
-    cfg.numAttrs = n_attr;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, p, tk, tv, cluster);
-    count_launch();
-    return e;
-}
-
 }  // namespace
+
+// block positions per 128-row query tile
+static int tc_kb_rows(const AttnParams &p) { return p.K < MROWS / p.G ? p.K : MROWS / p.G; }
+
+int tc_row_tiles(int G, int K)
+{
+    if (G < 1 || G > MROWS) return 0;
+    const int kb = K < MROWS / G ? K : MROWS / G;
+    return (K + kb - 1) / kb;
+}
 
 bool tc_path_supports(const AttnParams &p, int dtype)
 {
-    if (dtype != ORTHRUS_BF16 || p.d != HD || p.K > 64) return false;
+    if (dtype != ORTHRUS_BF16 || p.d != HD || p.K > TN || p.G > MROWS) return false;
     const unsigned long long rows = (unsigned long long)p.B * p.Hkv * p.capacity;
     return rows < 0x7fffffffull && encode_fn() != nullptr;
 }
 
-// Cluster size the kernel will use for a split count: all splits of a unit in one
-// cluster when there are at most 16, otherwise none (global partials + merge kernel).
-int tc_cluster_for_splits(int n_splits) { return n_splits <= 16 ? n_splits : 1; }
+int tc_ctas_per_sm() { return 2; }
+int tc_tile_positions() { return TN; }
 
-cudaError_t launch_attend_tc(const AttnParams &p, int tile, cudaStream_t st)
+cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st)
 {
-    const int cluster = tc_cluster_for_splits(p.n_splits);
-    int nsub = p.M <= 32 ? 4 : (p.M <= 64 ? 2 : 1);
-    while (nsub > 1 && (cluster * nsub > 32 || tile / nsub < 32)) nsub >>= 1;
-    if (tile == 64) {
-        return nsub >= 2 ? launch_one<64, 2>(p, cluster, st) : launch_one<64, 1>(p, cluster, st);
+    const int S = p.n_splits;
+    const int kb = tc_kb_rows(p);
+    TcMaps tm;
+    const unsigned long long rows = (unsigned long long)p.B * p.Hkv * p.capacity;
+    if (!get_map(p.k_cache, rows, 0, 0, TN, 0, &tm.k) || !get_map(p.v_cache, rows, 0, 0, TN, 0, &tm.v) ||
+        !get_map(p.q, p.Hq, p.K, p.B, p.G, kb, &tm.q) ||
+        !get_map(p.k_blk, p.Hkv, p.K, p.B, 1, TN, &tm.kb) || !get_map(p.v_blk, p.Hkv, p.K, p.B, 1, TN, &tm.vb))
+        return cudaErrorInvalidValue;
+    static std::once_flag once;
+    static cudaError_t cfg_err = cudaSuccess;
+    std::call_once(once, [] {
+        cfg_err = cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (cfg_err == cudaSuccess)
+            cfg_err = cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    });
+    if (cfg_err != cudaSuccess) return cfg_err;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(S, p.B * p.Hkv, (p.K + kb - 1) / kb);
+    cfg.blockDim = dim3(NTHREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (S > 1) {
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = S;
+        attr[n_attr].val.clusterDim.y = 1;
+        attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
     }
-    if (nsub == 4) return launch_one<128, 4>(p, cluster, st);
-    if (nsub == 2) return launch_one<128, 2>(p, cluster, st);
-    return launch_one<128, 1>(p, cluster, st);
+    if (!(flags & 2)) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n_attr;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attend_tc_kernel, p, tm, S, kb, flags & 1);
+    count_launch();
+    return e;
 }
 
 }  // namespace orthrus
-
-#ifdef ORTHRUS_TC_TRACE
-extern "C" int orthrus_debug_read_trace(unsigned long long *host, int n_words)
-{
-    return (int)cudaMemcpyFromSymbol(host, orthrus::g_trace, sizeof(unsigned long long) * n_words);
-}
-#endif

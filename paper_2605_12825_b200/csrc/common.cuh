@@ -54,8 +54,10 @@ bool mma_path_supports(const AttnParams &p, int dtype);
 cudaError_t launch_attend_mma(const AttnParams &p, cudaStream_t st);
 int mma_tile_positions();
 bool tc_path_supports(const AttnParams &p, int dtype);
-cudaError_t launch_attend_tc(const AttnParams &p, int tile, cudaStream_t st);
-int tc_cluster_for_splits(int n_splits);
+cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st);   // n_splits = cluster size
+int tc_row_tiles(int G, int K);          // 128-row query tiles per unit (0: group too wide)
+int tc_ctas_per_sm();
+int tc_tile_positions();
 cudaError_t launch_combine(const AttnParams &p, int dtype, cudaStream_t st);
 
 cudaError_t launch_consensus(const void *logits, int dtype, const int32_t *draft, int B, int K,
@@ -66,6 +68,11 @@ int consensus_segments(int B, int K, int V);
 cudaError_t launch_kv_append(const orthrus_layer_t &L, const void *k_blk, const void *v_blk,
                              const int32_t *n_commit, int update_len, int32_t *status,
                              cudaStream_t st);
+
+struct AppendLayer { void *k_cache, *v_cache; const void *k_blk, *v_blk; int32_t *cache_len; };
+cudaError_t launch_kv_append_layers(const orthrus_layer_t &shape, const AppendLayer *layers, int n_layers,
+                                    int32_t *const *len_arrays, int n_len_arrays,
+                                    const int32_t *n_commit, int32_t *status, cudaStream_t st);
 
 void count_launch(int n = 1);
 

@@ -39,7 +39,8 @@ def test_status_strings(lib):
 
 def _layer(lib, **kw):
     d = dict(batch=1, n_q_heads=8, n_kv_heads=2, head_dim=64, block=8, dtype=0, capacity=1024,
-             k_cache=0x1000, v_cache=0x2000, cache_len=0x3000, max_len_hint=512, softmax_scale=0.0)
+             k_cache=0x1000, v_cache=0x2000, cache_len=0x3000, max_len_hint=512, softmax_scale=0.0,
+             flags=0)
     d.update(kw)
     return lib.Layer(*[d[f[0]] for f in lib.Layer._fields_])
 
@@ -60,7 +61,7 @@ def test_workspace_query_and_plan(lib):
 @pytest.mark.parametrize("bad,code", [
     (dict(n_q_heads=7), 1), (dict(head_dim=48), 2), (dict(block=65), 2), (dict(dtype=5), 2),
     (dict(max_len_hint=1020), 3), (dict(k_cache=0), 1), (dict(k_cache=0x1008), 1),
-    (dict(softmax_scale=-1.0), 1),
+    (dict(softmax_scale=-1.0), 1), (dict(flags=8), 1),
 ])
 def test_attend_rejects_bad_descriptors_before_launch(lib, bad, code):
     L = _layer(lib, **bad)
@@ -72,7 +73,8 @@ def test_attend_rejects_bad_descriptors_before_launch(lib, bad, code):
 
 
 def test_null_and_small_workspace(lib):
-    L = _layer(lib, n_q_heads=32, n_kv_heads=8, head_dim=128, block=16, capacity=4160,
+    # head_dim 64 takes a path that keeps its split-KV partials in the workspace
+    L = _layer(lib, n_q_heads=32, n_kv_heads=8, head_dim=64, block=16, capacity=4160,
                max_len_hint=4096)
     f = lib.lib().orthrus_ar_verify_attend
     assert f(ctypes.byref(L), None, 0x5000, 0x6000, 0x7000, 0x8000, 1 << 30, None) == 1
