@@ -125,7 +125,7 @@ class DeviceState:
     """All tensors of the workload on one GPU, one set per layer (layers are distinct
     buffers, so every timed read of a long-prefix workload misses L2)."""
 
-    def __init__(self, wl: W.Workload, layers: int, dev: torch.device):
+    def __init__(self, wl: W.Workload, layers: int, dev: torch.device, layer_flags: int = 0):
         from paper_2605_12825_b200 import binding as B
         self.B, self.wl, self.layers, self.dev = B, wl, layers, dev
         self.lens_host = W.prefix_lengths(wl)
@@ -139,8 +139,10 @@ class DeviceState:
             t = {k: v.to(dev) for k, v in h.items()}
             self.t.append(t)
             self.host.append({k: v.pin_memory() for k, v in h.items() if "cache" not in k})
+            # in the step below no attention call directly follows a kernel that writes the
+            # cache or its lengths, which is what the flag promises
             self.layer.append(B.make_layer(t["k_cache"], t["v_cache"], self.cache_len,
-                                           wl.n_q_heads, wl.block, max_hint))
+                                           wl.n_q_heads, wl.block, max_hint, 0.0, layer_flags))
             self.out_d.append(torch.empty_like(t["q_diff"]))
             self.out_a.append(torch.empty_like(t["q_ar"]))
         self.ws = B.new_workspace(B.orthrus_attend_workspace_bytes(self.layer[0]))
@@ -181,12 +183,10 @@ class DeviceState:
                                         self.ar_argmax, self.next_anchor, self.cws)
 
     def phase_commit(self):
-        B = self.B
-        for l in range(self.layers):
-            t = self.t[l]
-            # all layers share one length array: only the last call grows it
-            B.orthrus_kv_append(self.layer[l], t["k_ar_blk"], t["v_ar_blk"], self.n_commit,
-                                l == self.layers - 1, self.ws)
+        # one launch commits the accepted rows of every layer; all layers share one length
+        # array, which grows once
+        self.B.orthrus_kv_append_layers(self.layer, [t["k_ar_blk"] for t in self.t],
+                                        [t["v_ar_blk"] for t in self.t], self.n_commit, True, self.ws)
         # the next step starts from the same prefix again (the appended bytes are identical
         # every step, so this rewinds the state exactly)
         self.cache_len.copy_(self.cache_len0)
@@ -242,7 +242,10 @@ def run_gpu(args):
 
     wl = W.CONFIGS[args.workload]
     layers = args.layers or wl.layers
-    st = DeviceState(wl, layers, dev)
+    flags = 0 if args.no_early_prefetch else B.LAYER_CACHE_QUIESCENT
+    if args.no_early_launch:
+        flags |= B.LAYER_NO_EARLY_LAUNCH
+    st = DeviceState(wl, layers, dev, flags)
     stream = torch.cuda.Stream(device=dev)
     phases = st.phases()
 
@@ -337,10 +340,12 @@ def run_gpu(args):
                    "kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "block": wl.block,
                    "prefix": [wl.prefix_min, wl.prefix_max], "vocab": wl.vocab, "layers": layers,
                    "step": "layers x (diffusion attend + AR verify attend) + consensus + "
-                           "layers x KV commit (+ rewind of cache_len)",
+                           "KV commit of all layers (+ rewind of cache_len)",
                    "l2": "inputs larger than L2 (distinct KV per layer)" if step_bytes > 2.5e8
                          else "L2-resident (reported, not a roofline workload)",
                    "cuda_graph": not args.no_graph, "attend_path": path,
+                   "early_launch": not args.no_early_launch,
+                   "early_cache_prefetch": not args.no_early_prefetch,
                    "multi_gpu": "replicas only"},
         "pct_of_hbm_peak": {"of_measured_%.0f" % peak if peak_kind == "measured" else
                             "of_fallback_%.0f" % peak: round(100 * kv_gbs / world / peak, 2),
@@ -471,6 +476,10 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.CONFIGS))
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-early-prefetch", action="store_true",
+                    help="do not set ORTHRUS_LAYER_CACHE_QUIESCENT on the layers")
+    ap.add_argument("--no-early-launch", action="store_true",
+                    help="launch the attention kernels in plain stream order")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()

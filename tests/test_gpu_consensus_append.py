@@ -141,3 +141,47 @@ def test_one_full_cycle_tiny_config():
     assert torch.equal(d["cache_len"].cpu(), ref["cache_len"])
     assert torch.equal(d["k_cache"].cpu().view(torch.int16), ref["k_cache"].view(torch.int16))
     assert torch.equal(d["v_cache"].cpu().view(torch.int16), ref["v_cache"].view(torch.int16))
+
+
+@pytest.mark.parametrize("update_len", [True, False])
+@pytest.mark.parametrize("shared_len", [True, False])
+def test_append_layers_bit_exact(update_len, shared_len):
+    """The multi-layer commit equals the oracle's commit applied layer by layer; a length
+    array shared by several layers grows once."""
+    b = binding()
+    L = 5
+    cases = [make_append_case(torch.bfloat16, seed=10 + l) for l in range(L)]
+    lens0 = torch.tensor([0, 17, 56], dtype=torch.int32)
+    n = torch.tensor([1, 8, 5], dtype=torch.int32)
+    ref = [{k: v.clone() for k, v in c.items()} for c in cases]
+    ref_lens = [lens0.clone() for _ in range(L)]
+    for l in range(L):
+        oracle.kv_append(ref[l]["k_cache"], ref[l]["v_cache"], ref_lens[l], ref[l]["k_blk"],
+                         ref[l]["v_blk"], n, update_len)
+    dev = [{k: v.cuda() for k, v in c.items()} for c in cases]
+    dl = [lens0.cuda()] * L if shared_len else [lens0.cuda() for _ in range(L)]
+    layers = [b.make_layer(d["k_cache"], d["v_cache"], dl[l], 4, 8) for l, d in enumerate(dev)]
+    ws = b.new_workspace(256)
+    b.orthrus_kv_append_layers(layers, [d["k_blk"] for d in dev], [d["v_blk"] for d in dev],
+                               n.cuda(), update_len, ws)
+    assert b.orthrus_read_status(ws) == 0
+    for l in range(L):
+        assert torch.equal(dev[l]["k_cache"].cpu().view(torch.int16), ref[l]["k_cache"].view(torch.int16))
+        assert torch.equal(dev[l]["v_cache"].cpu().view(torch.int16), ref[l]["v_cache"].view(torch.int16))
+        assert torch.equal(dl[l].cpu(), ref_lens[l])
+
+
+def test_append_layers_overflow_is_skipped_and_flagged():
+    b = binding()
+    cases = [make_append_case(torch.bfloat16, seed=20 + l) for l in range(2)]
+    lens = torch.tensor([0, 60, 10], dtype=torch.int32).cuda()      # 60 + 8 > 64
+    n = torch.tensor([2, 8, 9], dtype=torch.int32)                  # 9 > K
+    dev = [{k: v.cuda() for k, v in c.items()} for c in cases]
+    layers = [b.make_layer(d["k_cache"], d["v_cache"], lens, 4, 8) for d in dev]
+    ws = b.new_workspace(256)
+    b.orthrus_kv_append_layers(layers, [d["k_blk"] for d in dev], [d["v_blk"] for d in dev],
+                               n.cuda(), True, ws)
+    assert b.orthrus_read_status(ws) == b.DEV_APPEND_OVERFLOW
+    assert lens.cpu().tolist() == [2, 60, 10]
+    for d, c in zip(dev, cases):
+        assert torch.equal(d["k_cache"][1:].cpu().view(torch.int16), c["k_cache"][1:].view(torch.int16))
