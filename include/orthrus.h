@@ -158,6 +158,38 @@ orthrus_status_t orthrus_consensus_accept(const void *ar_logits, int32_t dtype,
         void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same consensus for callers that cannot hand over a workspace.  (The paper has no
+ * counterpart to this entry point; it exists for the embedding, not for the method.)
+ *
+ * Who needs it: code that runs where device memory may not be allocated - a plugin that
+ * is given its input and output buffers by a host runtime and is forbidden to call
+ * cudaMalloc (or any allocator built on it, a framework's caching allocator included),
+ * or a serving loop whose memory budget is fixed before it starts.  Such a caller can
+ * supply the logits, the drafts and the four result arrays, but has nowhere to get the
+ * scratch that the streaming argmax needs between its two kernels.
+ *
+ * Here that scratch is an array compiled into the library
+ * (ORTHRUS_STATIC_CONSENSUS_SCRATCH_BYTES of device memory on every GPU that loads the
+ * library, held until the process exits).  The call allocates nothing and frees nothing.
+ *   - Limit: batch * block * segments * 8 bytes must fit in the array, where segments is
+ *     the split of the vocabulary the library chooses (at most about 600 / (batch*block),
+ *     at least 1): in practice batch * block <= 8192 rows.  A larger problem returns
+ *     ORTHRUS_ERR_WORKSPACE and launches nothing; use orthrus_consensus_accept then.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside of any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the previous call
+ *     left in it.  Nothing has to be cleared (each call overwrites every entry it later
+ *     reads), but two calls that overlap on the GPU - different streams, or different
+ *     host threads - race on it and may both return wrong tokens.  Serialise them.
+ * Arguments, results and errors are otherwise those of orthrus_consensus_accept.
+ */
+#define ORTHRUS_STATIC_CONSENSUS_SCRATCH_BYTES 65536
+orthrus_status_t orthrus_consensus_accept_static(const void *ar_logits, int32_t dtype,
+        const int32_t *draft, int32_t batch, int32_t block, int32_t vocab,
+        int32_t *n_commit, int32_t *committed, int32_t *ar_argmax, int32_t *next_anchor,
+        void *stream);
+
+/*
  * KV commit (Figure 2(b); last paragraph of Section 3.3): for every sequence b,
  * KV head h and i < n_commit[b],
  *   k_cache[b][h][P_b + i] = k_ar_blk[b][i][h]   (likewise v),

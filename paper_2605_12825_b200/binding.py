@@ -24,6 +24,7 @@ EXPORTS = [
     "orthrus_attend_workspace_bytes", "orthrus_workspace_init",
     "orthrus_diffusion_block_attend", "orthrus_ar_verify_attend",
     "orthrus_consensus_workspace_bytes", "orthrus_consensus_accept",
+    "orthrus_consensus_accept_static",
     "orthrus_kv_append", "orthrus_kv_append_layers", "orthrus_read_status", "orthrus_set_path", "orthrus_last_path",
     "orthrus_launch_count", "orthrus_status_string", "orthrus_version",
 ]
@@ -70,6 +71,8 @@ def _load() -> ctypes.CDLL:
     lib.orthrus_consensus_workspace_bytes.argtypes = [i32, i32, i32]
     lib.orthrus_consensus_accept.restype = ctypes.c_int
     lib.orthrus_consensus_accept.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+    lib.orthrus_consensus_accept_static.restype = ctypes.c_int
+    lib.orthrus_consensus_accept_static.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.orthrus_kv_append.restype = ctypes.c_int
     lib.orthrus_kv_append.argtypes = [LP, vp, vp, vp, i32, vp, sz, vp]
     lib.orthrus_kv_append_layers.restype = ctypes.c_int
@@ -167,6 +170,22 @@ def orthrus_consensus_accept(ar_logits, draft, n_commit, committed, ar_argmax, n
         _ptr(ar_logits), dtype_code(ar_logits.dtype), _ptr(draft), B, K, V, _ptr(n_commit),
         _ptr(committed), _ptr(ar_argmax), _ptr(next_anchor), _ptr(workspace), workspace.numel(),
         _stream(stream)), "orthrus_consensus_accept")
+
+
+STATIC_CONSENSUS_SCRATCH_BYTES = 65536
+
+
+def orthrus_consensus_accept_static(ar_logits, draft, n_commit, committed, ar_argmax, next_anchor,
+                                    stream=None) -> None:
+    """Consensus without a caller-provided workspace: for callers that may not allocate
+    device memory.  The scratch is a fixed array inside the library, shared by all calls
+    on a device (calls that overlap on the GPU race on it).  Problems that need more than
+    STATIC_CONSENSUS_SCRATCH_BYTES of scratch raise OrthrusError (workspace too small)."""
+    B, K, V = ar_logits.shape
+    _check(_lib.orthrus_consensus_accept_static(
+        _ptr(ar_logits), dtype_code(ar_logits.dtype), _ptr(draft), B, K, V, _ptr(n_commit),
+        _ptr(committed), _ptr(ar_argmax), _ptr(next_anchor), _stream(stream)),
+        "orthrus_consensus_accept_static")
 
 
 def orthrus_kv_append(layer: Layer, k_ar_blk, v_ar_blk, n_commit, update_len: bool = True,

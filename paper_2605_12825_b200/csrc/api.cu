@@ -269,6 +269,30 @@ orthrus_status_t orthrus_consensus_accept(const void *ar_logits, int32_t dtype, 
     return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
 }
 
+orthrus_status_t orthrus_consensus_accept_static(const void *ar_logits, int32_t dtype,
+        const int32_t *draft, int32_t batch, int32_t block, int32_t vocab, int32_t *n_commit,
+        int32_t *committed, int32_t *ar_argmax, int32_t *next_anchor, void *stream)
+{
+    if (batch < 1 || block < 1 || vocab < 1) return ORTHRUS_ERR_INVALID_ARG;
+    if (dtype != ORTHRUS_BF16 && dtype != ORTHRUS_FP32) return ORTHRUS_ERR_UNSUPPORTED;
+    if (block > 1024 || (long long)batch * block > 65535) return ORTHRUS_ERR_UNSUPPORTED;
+    if (!ar_logits || !draft || !n_commit || !committed || !ar_argmax || !next_anchor)
+        return ORTHRUS_ERR_INVALID_ARG;
+    const size_t es = dtype == ORTHRUS_FP32 ? 4 : 2;
+    if ((reinterpret_cast<uintptr_t>(ar_logits) & (es - 1)) ||
+        ((reinterpret_cast<uintptr_t>(draft) | reinterpret_cast<uintptr_t>(n_commit) |
+          reinterpret_cast<uintptr_t>(committed) | reinterpret_cast<uintptr_t>(ar_argmax) |
+          reinterpret_cast<uintptr_t>(next_anchor)) & 3))
+        return ORTHRUS_ERR_INVALID_ARG;
+    // the built-in scratch has a fixed size: larger problems need the workspace variant
+    if (static_consensus_scratch_needed(batch, block, vocab) > (size_t)ORTHRUS_STATIC_CONSENSUS_SCRATCH_BYTES)
+        return ORTHRUS_ERR_WORKSPACE;
+    cudaError_t e = launch_consensus_static(ar_logits, dtype, draft, batch, block, vocab, n_commit,
+                                            committed, ar_argmax, next_anchor,
+                                            static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+}
+
 orthrus_status_t orthrus_kv_append(const orthrus_layer_t *layer, const void *k_ar_blk,
         const void *v_ar_blk, const int32_t *n_commit, int32_t update_len, void *workspace,
         size_t workspace_bytes, void *stream)

@@ -64,6 +64,10 @@ cudaError_t launch_consensus(const void *logits, int dtype, const int32_t *draft
                              int V, int32_t *n_commit, int32_t *committed, int32_t *ar_argmax,
                              int32_t *next_anchor, void *partials, int n_seg, cudaStream_t st);
 int consensus_segments(int B, int K, int V);
+size_t static_consensus_scratch_needed(int B, int K, int V);
+cudaError_t launch_consensus_static(const void *logits, int dtype, const int32_t *draft, int B, int K,
+                                    int V, int32_t *n_commit, int32_t *committed, int32_t *ar_argmax,
+                                    int32_t *next_anchor, cudaStream_t st);
 
 cudaError_t launch_kv_append(const orthrus_layer_t &L, const void *k_blk, const void *v_blk,
                              const int32_t *n_commit, int update_len, int32_t *status,

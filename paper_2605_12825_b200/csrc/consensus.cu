@@ -1,6 +1,7 @@
 // Greedy consensus: a streaming per-row argmax of the AR logits (16-byte loads, one
 // (value, index) pair per thread, warp-shuffle then shared-memory reduction with the
 // lowest index winning ties), followed by the sequential accept rule per sequence.
+#include <mutex>
 #include "common.cuh"
 
 namespace orthrus {
@@ -185,6 +186,55 @@ cudaError_t launch_consensus(const void *logits, int dtype, const int32_t *draft
                                                                     committed, ar_argmax, next_anchor);
     count_launch(2);
     return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- consensus without a workspace
+//
+// Scratch for orthrus_consensus_accept_static: the per-segment (value, index) pairs of the
+// streaming argmax.  It is part of the library image, so every GPU that loads the library
+// holds these bytes until the process exits.
+constexpr size_t kStaticScratchBytes = ORTHRUS_STATIC_CONSENSUS_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_consensus_scratch[kStaticScratchBytes];
+
+// In host code `g_consensus_scratch` only names the symbol; the address a kernel can use is
+// looked up once per device (with that device current) and remembered.
+static cudaError_t static_scratch_address(void **out)
+{
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static void *addr[kMaxDevices] = {};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_consensus_scratch);
+        if (e != cudaSuccess) return e;
+        if (!ptr) return cudaErrorInvalidSymbol;
+        addr[dev] = ptr;
+    }
+    *out = addr[dev];
+    return cudaSuccess;
+}
+
+size_t static_consensus_scratch_needed(int B, int K, int V)
+{
+    return (size_t)B * K * consensus_segments(B, K, V) * sizeof(ArgPart);
+}
+
+cudaError_t launch_consensus_static(const void *logits, int dtype, const int32_t *draft, int B, int K,
+                                    int V, int32_t *n_commit, int32_t *committed, int32_t *ar_argmax,
+                                    int32_t *next_anchor, cudaStream_t st)
+{
+    void *scratch = nullptr;
+    cudaError_t e = static_scratch_address(&scratch);
+    if (e != cudaSuccess) return e;
+    // every (row, segment) pair the second kernel reads is written by the first one in the
+    // same call, so nothing in the array has to start at zero
+    return launch_consensus(logits, dtype, draft, B, K, V, n_commit, committed, ar_argmax, next_anchor,
+                            scratch, consensus_segments(B, K, V), st);
 }
 
 }  // namespace orthrus
