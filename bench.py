@@ -68,6 +68,22 @@ def attend_bytes(wl: W.Workload, lens) -> int:
     return prefix + blk + qo
 
 
+def max_over_ranks(values, dist, device):
+    """Each rank times its own replica; the job's time is that of the slowest rank.
+    `dist` is torch.distributed with an initialised group, or None for one process."""
+    if dist is None:
+        return [float(v) for v in values]
+    tt = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return [float(v) for v in tt]
+
+
+def whole_job(per_rank_units: float, world: int, seconds: float) -> float:
+    """Replicas only: every rank processes the same number of units, the job's rate is all
+    of them over the slowest rank's time."""
+    return world * per_rank_units / seconds
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -316,14 +332,11 @@ def run_gpu(args):
         raise SystemExit(f"bench.py: device status word {status} after the timed region")
 
     ms_per_step = total_ms / args.steps
-    if dist is not None:
-        tt = torch.tensor([ms_per_step, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_per_step, e2e_ms = float(tt[0]), float(tt[1])
+    ms_per_step, e2e_ms = max_over_ranks([ms_per_step, e2e_ms], dist, dev)
 
     call_bytes = attend_bytes(wl, st.lens_host)
     step_bytes = call_bytes * 2 * layers
-    kv_gbs = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    kv_gbs = whole_job(step_bytes, world, ms_per_step * 1e-3) / 1e9
     tokens = int(n_commit.sum())
     peak, peak_kind = measured_peak()
     attend_ms = (phase_ms[0] + phase_ms[1]) / (2 * layers)
