@@ -86,8 +86,8 @@ static Plan make_plan(const orthrus_layer_t *L, bool tc)
     Plan pl;
     if (tc) {
         // The splits of a unit are the CTAs of one thread-block cluster (<= 16).  Few units:
-        // as many splits as still fit on the GPU in one wave.  Many units: enough CTAs for
-        // about three waves, so that sequences of unequal length pack well.
+        // as many splits as still fit on the GPU in one wave.  Many units: just enough CTAs
+        // to fill every slot once; sequences of unequal length are handed out longest first.
         const int tn = tc_tile_positions();
         const int units = L->batch * L->n_kv_heads * tc_row_tiles(L->n_q_heads / L->n_kv_heads, L->block);
         const int slots = tc_ctas_per_sm() * kNumSMs;
@@ -99,7 +99,9 @@ static Plan make_plan(const orthrus_layer_t *L, bool tc)
             const int min_tiles = env_int("ORTHRUS_MIN_CHUNK_TILES", 2);
             while (S < 16 && units * S * 2 <= slots && tiles / (S * 2) >= min_tiles) S *= 2;
         } else {
-            while (S < 16 && units * S < 3 * slots && tiles / (S * 2) >= 8) S *= 2;
+            // (a lone CTA streams slower than an SM's share of HBM, so the longest unit is
+            //  still split; many small CTAs would spend their time starting and merging)
+            while (S < 16 && units * S < slots && tiles / (S * 2) >= 8) S *= 2;
         }
         if (S > 16) S = 16;
         if (S > tiles) S = tiles;

@@ -3,9 +3,8 @@
 //
 // Work decomposition.  A unit is one (sequence, KV head); its query tile is the GQA
 // group times the block width, M = G*K logical rows (row r = i*G + g), padded to the
-// 128 rows of the MMA.  The S CTAs of a thread-block cluster share one unit: each takes
-// an equal share of the unit's 64-position prefix tiles, the last rank also takes the
-// tile of block keys.  Clusters are handed out longest sequence first, so that a ragged
+// 128 rows of the MMA.  The S CTAs of a thread-block cluster share one unit: the unit's
+// 64-position prefix tiles plus the tile of block keys are shared out evenly.  Clusters are handed out longest sequence first, so that a ragged
 // batch packs well onto the SMs.
 //
 // One CTA (192 threads, 112 KB of shared memory, 256 TMEM columns: two fit on an SM).
@@ -23,10 +22,15 @@
 // bf16 operands carry without loss, and the result is the exact softmax because the
 // same shift is used for the numerator and the denominator.
 //
+// Narrow units (M <= 64) load their query rows twice and run two independent softmax
+// streams over the two column halves of every tile, so that all 128 softmax threads work;
+// the two streams are folded together in shared memory before the merge.
+//
 // Merge.  Every CTA publishes its partial rows (max, sum, unnormalised O) in its own
 // shared memory; after a cluster barrier each CTA merges a slice of the rows straight
-// out of its peers' shared memory and writes the final bf16 rows.  No partial result
-// touches global memory and there is no second kernel.
+// out of its peers' shared memory (loads batched four rows deep, peers visited in a
+// rotated order) and writes the final bf16 rows.  No partial result touches global
+// memory and there is no second kernel.
 //
 // Programmatic dependent launch.  The kernel waits for the preceding kernel of the
 // stream (griddepcontrol.wait) before it reads anything that kernel may have written,
@@ -209,7 +213,23 @@ __device__ inline void tmem_st32(uint32_t taddr, const uint32_t *r) {
                    "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
                  : "memory");
 }
+__device__ inline void tmem_st16(uint32_t taddr, const uint32_t *r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]),
+                   "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]),
+                   "r"(r[14]), "r"(r[15])
+                 : "memory");
+}
 __device__ inline void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ inline float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+__device__ inline void named_bar_sync(int id, int n_threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
 __device__ inline float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -227,10 +247,19 @@ __device__ inline uint32_t sw_off(int r, int c, int sub_bytes) {
 
 struct TcMaps { CUtensorMap k, v, q, kb, vb; };
 
+// NSUB = 1: thread r of the softmax warps owns query row r and all 64 columns of a tile.
+// NSUB = 2 (units of at most 64 rows): the query rows are loaded twice, rows 64..127 being a
+// copy of rows 0..63; thread r works on logical row r % 64 and on columns [32*(r/64), +32)
+// of every tile only, so all 128 threads have work.  The two halves are independent
+// online-softmax streams (own max, own sum, own O row in TMEM) that are folded together
+// at the end exactly like the partial results of different CTAs.
+template <int NSUB>
 __global__ void __launch_bounds__(NTHREADS, 2)
 attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const int S, const int kb_rows,
                  const int quiescent)
 {
+    constexpr int W = TN / NSUB;              // score columns per softmax thread
+    constexpr int MPAD = MROWS / NSUB;        // logical rows per sub-stream
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t sbase = smem_u32(smem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + OFF_MISC + 8);
@@ -241,10 +270,10 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int rank = S > 1 ? (int)cluster_rank() : 0;
     const int order = blockIdx.y, rt = blockIdx.z;
-    // this row tile: kb_rows block positions x G heads
+    // this row tile: kb_rows block positions x G heads (at most MPAD rows)
     const int i0 = rt * kb_rows;
     const int rows_here = min(p.K - i0, kb_rows) * p.G;
-    const int n_act = (rows_here + 31) >> 5;                  // softmax warps with rows
+    const int n_act = NSUB * ((rows_here + 31) >> 5);         // softmax warps with rows
     const bool aligned = (sbase & 1023u) == 0;                // swizzled tiles need 1 KB alignment
 
     // ------------------------------------------------------------------ prologue
@@ -277,14 +306,14 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     // clusters are ordered longest prefix first (ties by sequence index)
     int b = order / p.Hkv;
     const int h = order % p.Hkv;
-    const long long len_hi = p.capacity - p.K;
+    const int len_hi = (int)(p.capacity - p.K);
     if (p.B > 1 && p.B <= 128) {
         const int want = b;
         for (int i = tid; i < p.B; i += NTHREADS) {
-            const long long Pi = min(max((long long)__ldg(p.cache_len + i), 0ll), len_hi);
+            const int Pi = min(max(__ldg(p.cache_len + i), 0), len_hi);
             int before = 0;
             for (int j = 0; j < p.B; ++j) {
-                const long long Pj = min(max((long long)__ldg(p.cache_len + j), 0ll), len_hi);
+                const int Pj = min(max(__ldg(p.cache_len + j), 0), len_hi);
                 before += (Pj > Pi) || (Pj == Pi && j < i);
             }
             if (before == want) *seq_slot = i;
@@ -295,14 +324,15 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     int P = p.cache_len[b];
     if (P < 0 || P > len_hi) {
         if (tid == 0 && rank == 0 && p.status) atomicOr(p.status, ORTHRUS_DEV_BAD_CACHE_LEN);
-        P = P < 0 ? 0 : (int)len_hi;
+        P = P < 0 ? 0 : len_hi;
     }
-    const int n_pre = (P + TN - 1) / TN;                      // prefix tiles of the unit
-    const int t0 = (int)((long long)rank * n_pre / S);
-    const int t1 = (int)((long long)(rank + 1) * n_pre / S);
-    const int n_mine = t1 - t0;                               // prefix tiles of this CTA
-    const bool owner = rank == S - 1;                         // also takes the block tile, last
-    const int n_tiles = n_mine + (owner ? 1 : 0);
+    // the unit's tiles: n_pre prefix tiles followed by the tile of block keys, shared out evenly
+    const uint32_t n_pre = (uint32_t)(P + TN - 1) / TN;
+    const uint32_t t0 = (uint32_t)rank * (n_pre + 1) / (uint32_t)S;
+    const uint32_t t1 = (uint32_t)(rank + 1) * (n_pre + 1) / (uint32_t)S;
+    const int n_tiles = (int)(t1 - t0);
+    const bool owner = rank == S - 1;                         // its last tile is the block tile
+    const int n_mine = n_tiles - (owner ? 1 : 0);             // prefix tiles of this CTA
     const bool active = n_tiles > 0 && aligned;
     const int row_base = (int)(((long long)b * p.Hkv + h) * p.capacity);   // row of position 0
 
@@ -315,7 +345,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
         mbar_expect_tx(fb, SLOT_BYTES);
         if (t < n_mine) {
             const CUtensorMap *m = is_v ? &tm.v : &tm.k;
-            const int row = row_base + (t0 + t) * TN;
+            const int row = row_base + ((int)t0 + t) * TN;
             tma_load_2d(dst, m, 0, row, fb);
             tma_load_2d(dst + SUB_BYTES, m, 64, row, fb);
         } else {                  // block tile: rows >= K are out of bounds and arrive as zeros
@@ -334,97 +364,132 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     }
     griddep_launch();
 
-    if (active && warp < n_act) {
-        // ------------------------------------------------------------------ softmax
+    if (warp < 4) {
         const int r = tid;
-        const bool valid = r < rows_here;
-        const int i_row = i0 + r / p.G;
+        const int sub = r / MPAD, Rl = r % MPAD;              // sub-stream, logical row in the tile
+        const bool valid = Rl < rows_here;
+        const bool warp_active = ((warp * 32) % MPAD) < rows_here;
+        const int i_row = i0 + Rl / p.G;
+        const int col0 = sub * W;
         const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-        const float sc = p.scale_log2;
         float m_run = -INFINITY, l_run = 0.f;
-        bool ok = true;
-        for (int t = 0; t < n_tiles; ++t) {
-            const int sb = t & 1;
-            ok = mbar_wait_warp(bar(BAR_SFULL + sb), (t >> 1) & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            uint32_t s[TN];
-            tmem_ld32(lane_base + TM_S + sb * TN, s);
-            tmem_ld32(lane_base + TM_S + sb * TN + 32, s + 32);
-            tmem_ld_wait();
-            // visible columns of this row in this tile
-            int lim;
-            if (t < n_mine) lim = min(TN, P - (t0 + t) * TN);
-            else lim = p.causal ? min(p.K, i_row + 1) : p.K;
-            if (!valid) lim = 0;
-            float mx = -INFINITY;
-            if (lim == TN) {
+        bool have_o = false;
+        if (active && warp_active) {
+            // -------------------------------------------------------------- softmax
+            const float sc = p.scale_log2;
+            const float2 sc2 = make_float2(sc, sc);
+            bool ok = true;
+            for (int t = 0; t < n_tiles; ++t) {
+                const int sb = t & 1;
+                ok = mbar_wait_warp(bar(BAR_SFULL + sb), (t >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t s[W];
 #pragma unroll
-                for (int j = 0; j < TN; ++j) mx = fmaxf(mx, __uint_as_float(s[j]));
-            } else {
+                for (int c = 0; c < W / 32; ++c) tmem_ld32(lane_base + TM_S + sb * TN + col0 + c * 32, s + c * 32);
+                tmem_ld_wait();
+                // visible columns of this row in this tile, then in this thread's column range
+                int lim;
+                if (t < n_mine) lim = min(TN, P - ((int)t0 + t) * TN);
+                else lim = p.causal ? min(p.K, i_row + 1) : p.K;
+                lim = valid ? min(W, max(0, lim - col0)) : 0;
+                float mx;
+                if (lim == W) {
+                    float m4[4];
 #pragma unroll
-                for (int j = 0; j < TN; ++j) if (j < lim) mx = fmaxf(mx, __uint_as_float(s[j]));
-            }
-            const float m_new = fmaxf(m_run, mx * sc);
-            const bool need = m_new > m_run + RESCALE_THRESHOLD;   // also the first finite maximum
-            if (__any_sync(0xffffffffu, need)) {
-                const float alpha = need ? ex2(m_run - m_new) : 1.f;
-                if (need) { m_run = m_new; l_run *= alpha; }
-                if (t > 0) {
-                    // O holds the products of tiles 0..t-1 and nothing is adding to it now
-                    ok = mbar_wait_warp(bar(BAR_PVDONE), (t - 1) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
+                    for (int q = 0; q < 4; ++q)
+                        m4[q] = max3(__uint_as_float(s[q]), __uint_as_float(s[q + 4]), __uint_as_float(s[q + 8]));
+#pragma unroll
+                    for (int j = 12; j + 8 <= W; j += 8)
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            m4[q] = max3(m4[q], __uint_as_float(s[j + q]), __uint_as_float(s[j + q + 4]));
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) m4[q] = fmaxf(m4[q], __uint_as_float(s[W - 4 + q]));
+                    mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+                } else {
+                    mx = -INFINITY;
+#pragma unroll
+                    for (int j = 0; j < W; ++j) if (j < lim) mx = fmaxf(mx, __uint_as_float(s[j]));
+                }
+                const float m_new = fmaxf(m_run, mx * sc);
+                const bool need = m_new > m_run + RESCALE_THRESHOLD;   // also the first finite maximum
+                if (__any_sync(0xffffffffu, need)) {
+                    const float alpha = need ? ex2(m_run - m_new) : 1.f;
+                    if (need) { m_run = m_new; l_run *= alpha; }
+                    if (t > 0) {
+                        // O holds the products of tiles 0..t-1 and nothing is adding to it now
+                        ok = mbar_wait_warp(bar(BAR_PVDONE), (t - 1) & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
 #pragma unroll 1
-                    for (int c4 = 0; c4 < HD / 32; ++c4) {
-                        uint32_t o[32];
-                        tmem_ld32(lane_base + TM_O + c4 * 32, o);
-                        tmem_ld_wait();
+                        for (int c4 = 0; c4 < HD / 32; ++c4) {
+                            uint32_t o[32];
+                            tmem_ld32(lane_base + TM_O + c4 * 32, o);
+                            tmem_ld_wait();
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-                        tmem_st32(lane_base + TM_O + c4 * 32, o);
+                            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+                            tmem_st32(lane_base + TM_O + c4 * 32, o);
+                        }
                     }
                 }
-            }
-            const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
-            uint32_t pk[TN / 2];
-            float lsum = 0.f;
-            if (lim == TN) {
+                const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
+                const float2 nm2 = make_float2(neg_m, neg_m);
+                uint32_t pk[W / 2];                            // this thread's probabilities, packed bf16
+                float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+                if (lim == W) {
 #pragma unroll
-                for (int j = 0; j < TN; j += 2) {
-                    const float p0 = ex2(fmaf(__uint_as_float(s[j]), sc, neg_m));
-                    const float p1 = ex2(fmaf(__uint_as_float(s[j + 1]), sc, neg_m));
-                    lsum += p0 + p1;
-                    pk[j >> 1] = pack_bf16(p0, p1);
-                }
-            } else {
+                    for (int j = 0; j < W; j += 4) {
+                        float2 a = __ffma2_rn(make_float2(__uint_as_float(s[j]), __uint_as_float(s[j + 1])), sc2, nm2);
+                        float2 c = __ffma2_rn(make_float2(__uint_as_float(s[j + 2]), __uint_as_float(s[j + 3])), sc2, nm2);
+                        a.x = ex2(a.x); a.y = ex2(a.y); c.x = ex2(c.x); c.y = ex2(c.y);
+                        acc0 = __fadd2_rn(acc0, a);
+                        acc1 = __fadd2_rn(acc1, c);
+                        pk[j >> 1] = pack_bf16(a.x, a.y);
+                        pk[(j >> 1) + 1] = pack_bf16(c.x, c.y);
+                    }
+                } else {
 #pragma unroll
-                for (int j = 0; j < TN; j += 2) {
-                    float p0 = ex2(fmaf(__uint_as_float(s[j]), sc, neg_m));
-                    float p1 = ex2(fmaf(__uint_as_float(s[j + 1]), sc, neg_m));
-                    if (j >= lim) p0 = 0.f;
-                    if (j + 1 >= lim) p1 = 0.f;
-                    lsum += p0 + p1;
-                    pk[j >> 1] = pack_bf16(p0, p1);
+                    for (int j = 0; j < W; j += 2) {
+                        float p0 = ex2(fmaf(__uint_as_float(s[j]), sc, neg_m));
+                        float p1 = ex2(fmaf(__uint_as_float(s[j + 1]), sc, neg_m));
+                        if (j >= lim) p0 = 0.f;
+                        if (j + 1 >= lim) p1 = 0.f;
+                        acc0.x += p0; acc0.y += p1;
+                        pk[j >> 1] = pack_bf16(p0, p1);
+                    }
                 }
+                l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
+                // P over the scores, 2 bf16 per column: the row's 32 packed columns are this
+                // thread's range and zeros for the range of the other sub-stream
+                if constexpr (NSUB == 1) {
+                    tmem_st32(lane_base + TM_S + sb * TN, pk);
+                } else {
+                    uint32_t zero[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) zero[j] = 0u;
+                    tmem_st16(lane_base + TM_S + sb * TN + sub * 16, pk);
+                    tmem_st16(lane_base + TM_S + sb * TN + (1 - sub) * 16, zero);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_PFULL + sb));
             }
-            l_run += lsum;
-            tmem_st32(lane_base + TM_S + sb * TN, pk);         // P over the scores, 2 bf16 per column
-            tmem_st_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_PFULL + sb));
+            // BAR_PVDONE cannot be used here: a parity wait cannot tell phase k from phase k-2, and
+            // by now the barrier may be one or two phases ahead of what this thread last observed
+            if (ok) ok = mbar_wait_warp(bar(BAR_ALLDONE), 0, abort_flag);
+            if (ok) tc_fence_after();
+            have_o = ok;
         }
-        // BAR_PVDONE cannot be used here: a parity wait cannot tell phase k from phase k-2, and
-        // by now the barrier may be one or two phases ahead of what this thread last observed
-        if (ok) ok = mbar_wait_warp(bar(BAR_ALLDONE), 0, abort_flag);
-        if (ok) {
-            tc_fence_after();
-            if (S == 1) {
-                // the whole unit was here: normalise and write the final rows
+
+        if (S == 1 && NSUB == 1) {
+            // ---------------------------------------------------------- direct output
+            // the whole unit was here: normalise and write the final rows
+            if (have_o) {
                 const float inv = 1.f / l_run;
                 __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.out) +
-                    (((long long)b * p.K + i_row) * p.Hq + h * p.G + (r % p.G)) * HD;
+                    (((long long)b * p.K + i_row) * p.Hq + h * p.G + (Rl % p.G)) * HD;
 #pragma unroll 1
                 for (int c4 = 0; c4 < HD / 32; ++c4) {
                     uint32_t o[32];
@@ -442,31 +507,80 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                         }
                     }
                 }
-            } else {
-                // publish the partial row; the ring is idle once the last product has landed
+            }
+        } else {
+            // ---------------------------------------------------------- publish partial rows
+            // every softmax thread puts its partial row (max, sum, unnormalised O straight out
+            // of TMEM) into this CTA's ring, which is idle once the last product has retired
+            if (have_o) {
 #pragma unroll 1
-                for (int c4 = 0; c4 < HD / 32; ++c4) {
-                    uint32_t o[32];
-                    tmem_ld32(lane_base + TM_O + c4 * 32, o);
+                for (int c2 = 0; c2 < HD / 64; ++c2) {
+                    uint32_t o[64];
+                    tmem_ld32(lane_base + TM_O + c2 * 64, o);
+                    tmem_ld32(lane_base + TM_O + c2 * 64 + 32, o + 32);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int c = 0; c < 8; ++c)
-                        *reinterpret_cast<uint4 *>(smem + OFF_OPART + r * 512 + (((c4 * 8 + c) ^ (r & 31)) << 4)) =
+                    for (int c = 0; c < 16; ++c)
+                        *reinterpret_cast<uint4 *>(smem + OFF_OPART + r * 512 + (((c2 * 16 + c) ^ (r & 31)) << 4)) =
                             make_uint4(o[c * 4], o[c * 4 + 1], o[c * 4 + 2], o[c * 4 + 3]);
                 }
+            }
+            if (valid && (have_o || !active)) {   // (threads without a row may get here before the ring is idle)
                 float *ml = reinterpret_cast<float *>(smem + OFF_ML);
-                ml[r * 2] = m_run;
-                ml[r * 2 + 1] = l_run;
+                ml[r * 2] = have_o ? m_run : -INFINITY;       // a CTA without tiles has empty rows
+                ml[r * 2 + 1] = have_o ? l_run : 0.f;
+            }
+            if constexpr (NSUB == 2) {
+                // fold the two sub-streams of a row together, in place in the first one's row:
+                // a warp per logical row, lane c holds output columns 4c..4c+3
+                named_bar_sync(1, 128);
+                float *ml = reinterpret_cast<float *>(smem + OFF_ML);
+                for (int R0 = warp; R0 < rows_here; R0 += 16) {   // four rows at a time, for latency
+                    float2 ma[4], mb[4];
+                    float4 va[4], vb[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int R = min(R0 + 4 * q, rows_here - 1), R2 = R + MPAD;
+                        ma[q] = *reinterpret_cast<const float2 *>(ml + R * 2);
+                        mb[q] = *reinterpret_cast<const float2 *>(ml + R2 * 2);
+                        va[q] = *reinterpret_cast<const float4 *>(smem + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4));
+                        vb[q] = *reinterpret_cast<const float4 *>(smem + OFF_OPART + R2 * 512 + ((lane ^ (R2 & 31)) << 4));
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int R = R0 + 4 * q;
+                        if (R < rows_here) {
+                            // a sub-stream without keys has sum 0 and its row was never written
+                            const bool ha = ma[q].y > 0.f, hb = mb[q].y > 0.f;
+                            const float mm = fmaxf(ha ? ma[q].x : -INFINITY, hb ? mb[q].x : -INFINITY);
+                            const float wa = ha ? ex2(ma[q].x - mm) : 0.f, wb = hb ? ex2(mb[q].x - mm) : 0.f;
+                            float4 o;
+                            o.x = wa * (ha ? va[q].x : 0.f) + wb * (hb ? vb[q].x : 0.f);
+                            o.y = wa * (ha ? va[q].y : 0.f) + wb * (hb ? vb[q].y : 0.f);
+                            o.z = wa * (ha ? va[q].z : 0.f) + wb * (hb ? vb[q].z : 0.f);
+                            o.w = wa * (ha ? va[q].w : 0.f) + wb * (hb ? vb[q].w : 0.f);
+                            *reinterpret_cast<float4 *>(smem + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4)) = o;
+                            if (lane == 0)
+                                *reinterpret_cast<float2 *>(ml + R * 2) =
+                                    make_float2(mm, wa * ma[q].y + wb * mb[q].y);
+                        }
+                    }
+                }
             }
         }
         tc_fence_before();
-    } else if (active && warp == 4) {
+    } else if (warp == 4) {
         // ------------------------------------------------------------------ producer
-        if (lane == 0) {
-            // the query rows of this tile: box = 64 columns x G heads x kb_rows positions
-            mbar_expect_tx(bar(BAR_QFULL), (uint32_t)(2 * 128 * p.G * kb_rows));
-            tma_load_4d(sbase + OFF_Q, &tm.q, 0, h * p.G, i0, b, bar(BAR_QFULL));
-            tma_load_4d(sbase + OFF_Q + QSUB_BYTES, &tm.q, 64, h * p.G, i0, b, bar(BAR_QFULL));
+        if (active && lane == 0) {
+            // the query rows of this tile: box = 64 columns x G heads x kb_rows positions,
+            // once per sub-stream
+            mbar_expect_tx(bar(BAR_QFULL), (uint32_t)(NSUB * 2 * 128 * p.G * kb_rows));
+#pragma unroll
+            for (int u = 0; u < NSUB; ++u) {
+                tma_load_4d(sbase + OFF_Q + u * MPAD * 128, &tm.q, 0, h * p.G, i0, b, bar(BAR_QFULL));
+                tma_load_4d(sbase + OFF_Q + QSUB_BYTES + u * MPAD * 128, &tm.q, 64, h * p.G, i0, b, bar(BAR_QFULL));
+            }
             bool ok = true;
             const int n_items = 2 * n_tiles;
             while (produced < n_items && ok) {
@@ -484,7 +598,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                 mbar_wait(bar(BAR_QFULL), 0, &dummy);
             }
         }
-    } else if (active && warp == 5) {
+    } else if (active) {
         // ------------------------------------------------------------------ MMA issue
         const uint32_t q_addr = sbase + OFF_Q;
         constexpr uint32_t IDESC_QK = make_idesc(TN, 0);      // A = Q, B = K tile, both K-major
@@ -513,7 +627,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             if (!mbar_wait_warp(bar(BAR_FULL + slot), (j / NSLOT) & 1, abort_flag)) return false;
             // a ragged prefix tile: V rows past the prefix may hold anything, and 0 * NaN would
             // poison the product, so they are cleared before the MMA reads them
-            const int nv = t < n_mine ? min(TN, P - (t0 + t) * TN) : TN;
+            const int nv = t < n_mine ? min(TN, P - ((int)t0 + t) * TN) : TN;
             if (nv < TN) {
                 unsigned char *vt = smem + OFF_RING + slot * SLOT_BYTES;
                 for (int e = lane; e < (TN - nv) * 16; e += 32) {
@@ -545,13 +659,9 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             if (t + 1 < n_tiles) ok = issue_qk(t + 1);
             if (ok) ok = issue_pv(t);
         }
-        // every MMA must have retired before the ring is reused and TMEM is freed
+        // every MMA must have retired before TMEM is freed
         if (ok) mbar_wait_warp(bar(BAR_ALLDONE), 0, abort_flag);
         tc_fence_before();
-    } else if (!active && S > 1 && tid < MROWS) {
-        float *ml = reinterpret_cast<float *>(smem + OFF_ML);
-        ml[tid * 2] = -INFINITY;              // a CTA without tiles publishes empty partial rows
-        ml[tid * 2 + 1] = 0.f;
     }
 
     // ---------------------------------------------------------------------- merge
@@ -560,51 +670,84 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     if (warp == 5)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TM_COLS) : "memory");
     if (tid == 0 && *abort_flag && p.status) atomicOr(p.status, ORTHRUS_DEV_WAIT_TIMEOUT);
-    if (S == 1) return;
-    cluster_sync_all();
+    if (S == 1 && NSUB == 1) return;
+    if (S > 1) cluster_sync_all();                            // every CTA's partial rows are in place
 
-    // rank k merges rows k, k+S, ...: lane j holds the weight of partial j, every lane four
-    // output columns
-    for (int Rl = rank + S * warp; Rl < rows_here; Rl += S * (NTHREADS / 32)) {
-        float mj = -INFINITY, lj = 0.f;
-        if (lane < S) {
-            const float2 v = ld_cluster_f2(map_to_rank(sbase + OFF_ML + Rl * 8, lane));
-            mj = v.x; lj = v.y;
-        }
-        float mmax = mj;
+    // Row R of the tile is merged and written by cluster rank R % S, which reads the row's S
+    // partial results out of its peers' shared memory: a warp per row, lane j holds the weight
+    // of the partial of rank j, every lane four output columns.  Rows are taken four at a time
+    // and all their loads are issued before the first is used, so that a warp pays the
+    // latency of the SM-to-SM path once per batch, not once per load.
+    const int my_rows = rank < rows_here ? (rows_here - rank + S - 1) / S : 0;
+    constexpr int NWARPS = NTHREADS / 32;
+    for (int s0 = warp; s0 < my_rows; s0 += 4 * NWARPS) {
+        float mj[4], lj[4];
 #pragma unroll
-        for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
-        const float wj = (lj > 0.f) ? ex2(mj - mmax) : 0.f;
-        float L = wj * lj;
-#pragma unroll
-        for (int off = 16; off; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
-        const uint32_t local = sbase + OFF_OPART + Rl * 512 + ((lane ^ (Rl & 31)) << 4);
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int j0 = 0; j0 < S; j0 += 8) {
-            float4 v[8];
-            float w[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int j = min(j0 + u, S - 1);
-                w[u] = (j0 + u < S) ? __shfl_sync(0xffffffffu, wj, j) : 0.f;
-                v[u] = ld_cluster_f4(map_to_rank(local, j));
+        for (int q = 0; q < 4; ++q) {
+            const int R = rank + min(s0 + q * NWARPS, my_rows - 1) * S;
+            mj[q] = -INFINITY; lj[q] = 0.f;
+            if (lane < S && s0 + q * NWARPS < my_rows) {
+                const uint32_t a = sbase + OFF_ML + R * 8;
+                const float2 v = ld_cluster_f2(S > 1 ? map_to_rank(a, lane) : a);
+                mj[q] = v.x; lj[q] = v.y;
             }
+        }
+        float wj[4], L[4];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                // an empty partial has weight 0 and unwritten rows: keep them out of the sum
-                if (w[u] != 0.f) {
-                    acc.x = fmaf(w[u], v[u].x, acc.x); acc.y = fmaf(w[u], v[u].y, acc.y);
-                    acc.z = fmaf(w[u], v[u].z, acc.z); acc.w = fmaf(w[u], v[u].w, acc.w);
+        for (int q = 0; q < 4; ++q) {
+            float mmax = mj[q];
+#pragma unroll
+            for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
+            wj[q] = (lj[q] > 0.f) ? ex2(mj[q] - mmax) : 0.f;
+            L[q] = wj[q] * lj[q];
+#pragma unroll
+            for (int off = 16; off; off >>= 1) L[q] += __shfl_xor_sync(0xffffffffu, L[q], off);
+        }
+        float4 acc[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int j0 = 0; j0 < S; j0 += 4) {
+            float4 v[4][4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int R = rank + min(s0 + q * NWARPS, my_rows - 1) * S;
+                const uint32_t a = sbase + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    // every CTA starts with its own partial, so that at any moment the CTAs of
+                    // the cluster read from different peers
+                    const int j = (min(j0 + u, S - 1) + rank) % S;
+                    if (s0 + q * NWARPS < my_rows) v[q][u] = ld_cluster_f4(S > 1 ? map_to_rank(a, j) : a);
                 }
             }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int j = (min(j0 + u, S - 1) + rank) % S;
+                    const float w = (j0 + u < S) ? __shfl_sync(0xffffffffu, wj[q], j) : 0.f;
+                    // a partial without keys has weight 0 and its row was never written
+                    if (w != 0.f) {
+                        acc[q].x = fmaf(w, v[q][u].x, acc[q].x); acc[q].y = fmaf(w, v[q][u].y, acc[q].y);
+                        acc[q].z = fmaf(w, v[q][u].z, acc[q].z); acc[q].w = fmaf(w, v[q][u].w, acc[q].w);
+                    }
+                }
         }
-        const int i = i0 + Rl / p.G, g = Rl % p.G;
-        const float inv = 1.f / L;
-        uint2 *dst = reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) +
-                     (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD);
-        dst[lane] = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int slot = s0 + q * NWARPS;
+            if (slot < my_rows) {
+                const int R = rank + slot * S;
+                const int i = i0 + R / p.G, g = R % p.G;
+                const float inv = 1.f / L[q];
+                uint2 *dst = reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) +
+                             (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD);
+                dst[lane] = make_uint2(pack_bf16(acc[q].x * inv, acc[q].y * inv),
+                                       pack_bf16(acc[q].z * inv, acc[q].w * inv));
+            }
+        }
     }
-    cluster_sync_all();     // peers may still be reading this CTA's rows
+    if (S > 1) cluster_sync_all();     // peers may still be reading this CTA's rows
 }
 
 // ---------------------------------------------------------------------------- host side
@@ -677,13 +820,15 @@ bool get_map(const void *ptr, unsigned long long d1, unsigned long long d2, unsi
 
 }  // namespace
 
-// block positions per 128-row query tile
-static int tc_kb_rows(const AttnParams &p) { return p.K < MROWS / p.G ? p.K : MROWS / p.G; }
+// Sub-streams per query row: 2 when a unit has at most 64 rows, else 1.
+static int tc_nsub(int G, int K) { return G * K <= 64 ? 2 : 1; }
+// block positions per query tile of 128 / nsub rows
+static int tc_kb_rows(int G, int K, int nsub) { return K < (MROWS / nsub) / G ? K : (MROWS / nsub) / G; }
 
 int tc_row_tiles(int G, int K)
 {
     if (G < 1 || G > MROWS) return 0;
-    const int kb = K < MROWS / G ? K : MROWS / G;
+    const int kb = tc_kb_rows(G, K, tc_nsub(G, K));
     return (K + kb - 1) / kb;
 }
 
@@ -697,22 +842,16 @@ bool tc_path_supports(const AttnParams &p, int dtype)
 int tc_ctas_per_sm() { return 2; }
 int tc_tile_positions() { return TN; }
 
-cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st)
+template <int NSUB>
+static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int flags, cudaStream_t st)
 {
     const int S = p.n_splits;
-    const int kb = tc_kb_rows(p);
-    TcMaps tm;
-    const unsigned long long rows = (unsigned long long)p.B * p.Hkv * p.capacity;
-    if (!get_map(p.k_cache, rows, 0, 0, TN, 0, &tm.k) || !get_map(p.v_cache, rows, 0, 0, TN, 0, &tm.v) ||
-        !get_map(p.q, p.Hq, p.K, p.B, p.G, kb, &tm.q) ||
-        !get_map(p.k_blk, p.Hkv, p.K, p.B, 1, TN, &tm.kb) || !get_map(p.v_blk, p.Hkv, p.K, p.B, 1, TN, &tm.vb))
-        return cudaErrorInvalidValue;
     static std::once_flag once;
     static cudaError_t cfg_err = cudaSuccess;
     std::call_once(once, [] {
-        cfg_err = cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        cfg_err = cudaFuncSetAttribute(attend_tc_kernel<NSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (cfg_err == cudaSuccess)
-            cfg_err = cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            cfg_err = cudaFuncSetAttribute(attend_tc_kernel<NSUB>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     });
     if (cfg_err != cudaSuccess) return cfg_err;
     cudaLaunchConfig_t cfg = {};
@@ -729,16 +868,30 @@ cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st)
         attr[n_attr].val.clusterDim.z = 1;
         ++n_attr;
     }
-    if (!(flags & 2)) {
+    if (!(flags & ORTHRUS_LAYER_NO_EARLY_LAUNCH)) {
         attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
         ++n_attr;
     }
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, attend_tc_kernel, p, tm, S, kb, flags & 1);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attend_tc_kernel<NSUB>, p, tm, S, kb,
+                                       (flags & ORTHRUS_LAYER_CACHE_QUIESCENT) ? 1 : 0);
     count_launch();
     return e;
+}
+
+cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st)
+{
+    const int nsub = tc_nsub(p.G, p.K);
+    const int kb = tc_kb_rows(p.G, p.K, nsub);
+    TcMaps tm;
+    const unsigned long long rows = (unsigned long long)p.B * p.Hkv * p.capacity;
+    if (!get_map(p.k_cache, rows, 0, 0, TN, 0, &tm.k) || !get_map(p.v_cache, rows, 0, 0, TN, 0, &tm.v) ||
+        !get_map(p.q, p.Hq, p.K, p.B, p.G, kb, &tm.q) ||
+        !get_map(p.k_blk, p.Hkv, p.K, p.B, 1, TN, &tm.kb) || !get_map(p.v_blk, p.Hkv, p.K, p.B, 1, TN, &tm.vb))
+        return cudaErrorInvalidValue;
+    return nsub == 2 ? launch_tc<2>(p, tm, kb, flags, st) : launch_tc<1>(p, tm, kb, flags, st);
 }
 
 }  // namespace orthrus
