@@ -22,9 +22,9 @@
 // bf16 operands carry without loss, and the result is the exact softmax because the
 // same shift is used for the numerator and the denominator.
 //
-// Narrow units (M <= 64) load their query rows twice and run two independent softmax
-// streams over the two column halves of every tile, so that all 128 softmax threads work;
-// the two streams are folded together in shared memory before the merge.
+// Narrow units (M <= 64) can optionally load their query rows twice and run two independent
+// softmax streams over the two column halves of every tile, so that all 128 softmax
+// threads work; the two streams are folded together in shared memory before the merge.
 //
 // Merge.  Every CTA publishes its partial rows (max, sum, unnormalised O) in its own
 // shared memory; after a cluster barrier each CTA merges a slice of the rows straight
@@ -42,6 +42,7 @@
 // the status word, drains the copies it armed, still takes part in the cluster barriers,
 // frees its TMEM and returns.
 #include <cuda.h>
+#include <cstdlib>
 #include <mutex>
 #include <unordered_map>
 #include "common.cuh"
@@ -680,6 +681,45 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     // latency of the SM-to-SM path once per batch, not once per load.
     const int my_rows = rank < rows_here ? (rows_here - rank + S - 1) / S : 0;
     constexpr int NWARPS = NTHREADS / 32;
+    if (my_rows <= NWARPS) {
+        // at most one row per warp: all of the row's partial results are requested at once
+        if (warp < my_rows) {
+            const int R = rank + warp * S;
+            float mj = -INFINITY, lj = 0.f;
+            if (lane < S) {
+                const uint32_t a = sbase + OFF_ML + R * 8;
+                const float2 v = ld_cluster_f2(S > 1 ? map_to_rank(a, lane) : a);
+                mj = v.x; lj = v.y;
+            }
+            const uint32_t a = sbase + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4);
+            float4 v[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u)
+                if (u < S) v[u] = ld_cluster_f4(S > 1 ? map_to_rank(a, u) : a);
+            float mmax = mj;
+#pragma unroll
+            for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
+            const float wj = (lj > 0.f) ? ex2(mj - mmax) : 0.f;
+            float L = wj * lj;
+#pragma unroll
+            for (int off = 16; off; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                const float w = (u < S) ? __shfl_sync(0xffffffffu, wj, u) : 0.f;
+                // a partial without keys has weight 0 and its row was never written
+                if (w != 0.f) {
+                    acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
+                    acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);
+                }
+            }
+            const int i = i0 + R / p.G, g = R % p.G;
+            const float inv = 1.f / L;
+            uint2 *dst = reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) +
+                         (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD);
+            dst[lane] = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+        }
+    } else
     for (int s0 = warp; s0 < my_rows; s0 += 4 * NWARPS) {
         float mj[4], lj[4];
 #pragma unroll
@@ -821,7 +861,14 @@ bool get_map(const void *ptr, unsigned long long d1, unsigned long long d2, unsi
 }  // namespace
 
 // Sub-streams per query row: 2 when a unit has at most 64 rows, else 1.
-static int tc_nsub(int G, int K) { return G * K <= 64 ? 2 : 1; }
+// Sub-streams per query row.  Two sub-streams halve the softmax time of a tile for units of
+// at most 64 rows, but their extra fold step costs more than that at the tile counts per
+// CTA measured so far, so they are opt-in (ORTHRUS_TC_NSUB=2) and one is the default.
+static int tc_nsub(int G, int K)
+{
+    static const int forced = [] { const char *e = getenv("ORTHRUS_TC_NSUB"); return e ? atoi(e) : 0; }();
+    return (forced == 2 && G * K <= 64) ? 2 : 1;
+}
 // block positions per query tile of 128 / nsub rows
 static int tc_kb_rows(int G, int K, int nsub) { return K < (MROWS / nsub) / G ? K : (MROWS / nsub) / G; }
 
