@@ -1,0 +1,116 @@
+"""End-to-end generation loop on a random-initialised decoder (the shape of the fifth
+benchmark configuration, scaled down): prefill, then repeated block-K draft / verify /
+consensus / commit through the C ABI, with drafts forced to agree with the AR greedy
+trajectory at a set rate so that acceptance is controlled.
+
+Checks: (1) the lossless guarantee of Section 3.3 - the committed stream equals plain
+greedy decoding (the same library path at block width 1) token for token in the fp32
+test mode; in bf16, block-K verification and width-1 decoding round differently, so
+equality is required up to the first position whose top-2 logit gap in the width-1 run
+is below a stated epsilon; (2) every cycle's consensus equals the oracle's on the GPU's
+own logits, bit for bit; (3) 1 <= n <= K and the cache length grows by n."""
+import pytest
+import torch
+
+import oracle
+from _decoder_harness import Decoder
+from _gpu_util import binding
+
+pytestmark = pytest.mark.gpu
+
+
+def greedy_trajectory(dec, anchor, n_new):
+    """Width-1 decoding with the AR view: returns tokens [B][n_new] and top-2 gaps."""
+    b = dec.b
+    B = anchor.shape[0]
+    i32 = dict(dtype=torch.int32, device="cuda")
+    outs = [torch.zeros(B, **i32), torch.zeros(B, 1, **i32), torch.zeros(B, 1, **i32), torch.zeros(B, **i32)]
+    cws = b.new_workspace(b.orthrus_consensus_workspace_bytes(B, 1, dec.V))
+    toks, gaps = [], []
+    draft = torch.zeros(B, 1, **i32)
+    for _ in range(n_new):
+        logits, ks, vs = dec.forward_block(anchor.view(B, 1), "ar", 1)
+        b.orthrus_consensus_accept(logits, draft, *outs, cws)
+        top2 = logits.float().topk(2, dim=-1).values[:, 0]
+        gaps.append((top2[:, 0] - top2[:, 1]).cpu())
+        dec.commit(ks, vs, outs[0], 1)
+        anchor = outs[3].clone()
+        toks.append(anchor.cpu())
+    return torch.stack(toks, 1), torch.stack(gaps, 1)
+
+
+def run_loop(dtype, layers, hidden, n_q, n_kv, d, ffn, vocab, B, T, K, n_new, rate, eps):
+    b = binding()
+    b.orthrus_set_path("auto")
+    cap = T + n_new + 2 * K + 8
+    g = torch.Generator().manual_seed(11)
+    prompt = torch.randint(0, vocab, (B, T), generator=g).cuda()
+
+    ref = Decoder(b, layers, hidden, n_q, n_kv, d, ffn, vocab, dtype, B, cap, K, seed=3)
+    anchor0 = ref.prefill(prompt)
+    traj, gaps = greedy_trajectory(ref, anchor0, n_new + K)
+
+    dec = Decoder(b, layers, hidden, n_q, n_kv, d, ffn, vocab, dtype, B, cap, K, seed=3,
+                  flags=b.LAYER_CACHE_QUIESCENT)
+    anchor = dec.prefill(prompt)
+    assert torch.equal(anchor.cpu(), anchor0.cpu())
+    streams = [[] for _ in range(B)]
+    cycles, total = 0, 0
+    while min(len(s) for s in streams) < n_new:
+        done = torch.tensor([len(s) for s in streams])
+        # forced drafts: the trajectory token with probability `rate`, else a uniform token
+        idx = (done.view(B, 1) + torch.arange(K)).clamp(max=traj.shape[1] - 1)
+        want = torch.gather(traj, 1, idx)
+        coin = torch.rand(B, K, generator=g) < rate
+        draft = torch.where(coin, want, torch.randint(0, vocab, (B, K), generator=g, dtype=torch.int32))
+        draft = draft.to(torch.int32).cuda()
+        len_before = dec.cache_len.cpu().clone()
+        # forward pass 1: the diffusion view over [anchor, mask x (K-1)]
+        blk = torch.full((B, K), vocab, dtype=torch.int32, device="cuda")
+        blk[:, 0] = anchor
+        d_logits, _, _ = dec.forward_block(blk, "diff", K)
+        assert torch.isfinite(d_logits.float()).all()
+        # forward pass 2: the AR view over [anchor, draft_1 .. draft_{K-1}]
+        ar_in = torch.cat([anchor.view(B, 1), draft[:, :K - 1]], dim=1)
+        logits, ks, vs = dec.forward_block(ar_in, "ar", K)
+        b.orthrus_consensus_accept(logits, draft, dec.n_commit, dec.committed, dec.ar_argmax,
+                                   dec.next_anchor, dec.cws)
+        rn, rcom, rarg, rnxt = oracle.consensus_accept(logits.cpu(), draft.cpu())
+        assert torch.equal(dec.n_commit.cpu(), rn) and torch.equal(dec.committed.cpu(), rcom)
+        assert torch.equal(dec.ar_argmax.cpu(), rarg) and torch.equal(dec.next_anchor.cpu(), rnxt)
+        assert int(rn.min()) >= 1 and int(rn.max()) <= K
+        dec.commit(ks, vs, dec.n_commit, K)
+        assert torch.equal(dec.cache_len.cpu(), len_before + rn)
+        assert b.orthrus_read_status(dec.ws) == 0
+        for s in range(B):
+            streams[s].extend(rcom[s, :int(rn[s])].tolist())
+        anchor = dec.next_anchor.clone()
+        cycles += 1
+        total += int(rn.sum())
+    # lossless: equal to greedy decoding, up to a near tie of the width-1 run (bf16 only)
+    near_ties = 0
+    for s in range(B):
+        got = streams[s][:n_new]
+        exp = traj[s, :n_new].tolist()
+        for i, (x, y) in enumerate(zip(got, exp)):
+            if x != y:
+                assert float(gaps[s, i]) < eps, (s, i, x, y, float(gaps[s, i]))
+                near_ties += 1
+                break
+    return total / (cycles * B), near_ties
+
+
+def test_lossless_generation_fp32_reduced_model():
+    mean_n, ties = run_loop(torch.float32, layers=2, hidden=128, n_q=4, n_kv=2, d=32, ffn=256,
+                            vocab=500, B=3, T=40, K=8, n_new=40, rate=0.65, eps=1e-4)
+    assert ties == 0
+    assert 1.5 < mean_n < 4.5          # E[n] = (1 - p^K) / (1 - p) = 2.77 for p = 0.65, K = 8
+
+
+def test_generation_bf16_tcgen05_shapes():
+    """head_dim 128, G = 4, K = 16 (M = 64): the shapes of the benchmark's decoder configuration."""
+    mean_n, ties = run_loop(torch.bfloat16, layers=3, hidden=512, n_q=8, n_kv=2, d=128, ffn=1024,
+                            vocab=2000, B=4, T=300, K=16, n_new=48, rate=0.65, eps=0.25)
+    assert ties <= 2
+    assert 1.5 < mean_n < 4.5
+    assert binding().orthrus_last_path() == "tcgen05"
