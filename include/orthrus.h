@@ -104,9 +104,8 @@ enum {
 /*
  * Bytes of workspace the two attention calls (and orthrus_kv_append) need for
  * this layer shape: a 256-byte header holding the status word, followed by the
- * split-KV partial results of the kernel paths that keep them in global memory
- * (the tcgen05 path merges its splits on chip and uses the header only).
- * Returns 0 for an invalid descriptor.
+ * split-KV partial results (written and read back inside one call; they are meant
+ * to stay in L2).  Returns 0 for an invalid descriptor.
  */
 size_t orthrus_attend_workspace_bytes(const orthrus_layer_t *layer);
 

@@ -133,9 +133,12 @@ static Plan make_plan(const orthrus_layer_t *L, bool tc)
 static size_t partial_bytes(const orthrus_layer_t *L, const Plan &pl, size_t *ml_off, bool tc = false)
 {
     if (ml_off) *ml_off = 0;
-    if (tc || pl.n_splits == 1) return 0;      // the tcgen05 path merges its splits on chip
-    const size_t units = (size_t)L->batch * L->n_kv_heads;
-    const size_t M = (size_t)(L->n_q_heads / L->n_kv_heads) * L->block;
+    if (pl.n_splits == 1 || (tc && pl.n_splits <= tc_dsmem_max_cluster())) return 0;
+    // the tcgen05 path keeps one 128-row partial tile per CTA (clusters too large for the
+    // on-chip exchange only)
+    const size_t units = (size_t)L->batch * L->n_kv_heads *
+                         (tc ? tc_row_tiles(L->n_q_heads / L->n_kv_heads, L->block) : 1);
+    const size_t M = tc ? 128 : (size_t)(L->n_q_heads / L->n_kv_heads) * L->block;
     const size_t o_bytes = units * pl.n_splits * M * L->head_dim * sizeof(float);
     const size_t ml_bytes = units * pl.n_splits * M * 2 * sizeof(float);
     if (ml_off) *ml_off = o_bytes;

@@ -26,11 +26,14 @@
 // softmax streams over the two column halves of every tile, so that all 128 softmax
 // threads work; the two streams are folded together in shared memory before the merge.
 //
-// Merge.  Every CTA publishes its partial rows (max, sum, unnormalised O) in its own
-// shared memory; after a cluster barrier each CTA merges a slice of the rows straight
-// out of its peers' shared memory (loads batched four rows deep, peers visited in a
-// rotated order) and writes the final bf16 rows.  No partial result touches global
-// memory and there is no second kernel.
+// Merge.  Every softmax thread puts its partial row (max, sum, unnormalised O straight out
+// of TMEM) into its CTA's idle ring.  Row r of the tile is merged and written by cluster
+// rank r % S.  Clusters of up to 8 CTAs read the rows they merge straight out of their
+// peers' shared memory, between two cluster barriers.  Larger clusters go through the
+// workspace (L2): each CTA copies its rows out with 512-byte coalesced stores, one cluster
+// barrier publishes them, the owners read them back and a CTA leaves as soon as its own
+// rows are written; for a 16-CTA all-to-all the SM-to-SM path was measured to be slower
+// than that.  There is no second kernel.
 //
 // Programmatic dependent launch.  The kernel waits for the preceding kernel of the
 // stream (griddepcontrol.wait) before it reads anything that kernel may have written,
@@ -76,6 +79,7 @@ static_assert(NUM_BARS <= 24, "barrier area");
 
 constexpr uint32_t TM_O = 0, TM_S = 128, TM_COLS = 256;   // TMEM column map
 constexpr float RESCALE_THRESHOLD = 8.f;                  // log2 units
+constexpr int kDsmemMaxCluster = 8;                       // larger clusters exchange partials through L2
 
 __device__ inline uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -247,6 +251,96 @@ __device__ inline uint32_t sw_off(int r, int c, int sub_bytes) {
 }
 
 struct TcMaps { CUtensorMap k, v, q, kb, vb; };
+
+// Split merge.  Row R of a tile is merged and written by cluster rank R % S: a warp per row,
+// lane j holds the weight of the partial result of rank j, every lane four output columns.
+// load_ml(j, R) returns (max, sum) of rank j's partial row R, load_o(j, R) this lane's four
+// columns of it.  The loads of a batch are all issued before the first is used.
+template <class LoadML, class LoadO, class Store>
+__device__ inline void merge_rows(int S, int rank, int my_rows, int warp, int lane, int n_warps,
+                                  LoadML load_ml, LoadO load_o, Store store)
+{
+    if (my_rows <= n_warps) {
+        // at most one row per warp: all of the row's partial results are requested at once
+        if (warp < my_rows) {
+            const int R = rank + warp * S;
+            float mj = -INFINITY, lj = 0.f;
+            if (lane < S) { const float2 t2 = load_ml(lane, R); mj = t2.x; lj = t2.y; }
+            float4 v[16];
+#pragma unroll
+            for (int u = 0; u < 16; ++u)
+                if (u < S) v[u] = load_o(u, R);
+            float mmax = mj;
+#pragma unroll
+            for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
+            const float wj = (lj > 0.f) ? ex2(mj - mmax) : 0.f;
+            float L = wj * lj;
+#pragma unroll
+            for (int off = 16; off; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 16; ++u) {
+                const float w = (u < S) ? __shfl_sync(0xffffffffu, wj, u) : 0.f;
+                // a partial without keys has weight 0 and its row was never written
+                if (w != 0.f) {
+                    acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
+                    acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);
+                }
+            }
+            store(R, acc, 1.f / L);
+        }
+        return;
+    }
+    for (int s0 = warp; s0 < my_rows; s0 += 4 * n_warps) {
+        float mj[4], lj[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int R = rank + min(s0 + q * n_warps, my_rows - 1) * S;
+            mj[q] = -INFINITY; lj[q] = 0.f;
+            if (lane < S && s0 + q * n_warps < my_rows) { const float2 t2 = load_ml(lane, R); mj[q] = t2.x; lj[q] = t2.y; }
+        }
+        float4 acc[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        float wj[4] = {0.f, 0.f, 0.f, 0.f}, L[4] = {1.f, 1.f, 1.f, 1.f};
+        for (int j0 = 0; j0 < S; j0 += 4) {
+            float4 v[4][4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int R = rank + min(s0 + q * n_warps, my_rows - 1) * S;
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (j0 + u < S && s0 + q * n_warps < my_rows) v[q][u] = load_o(j0 + u, R);
+            }
+            if (j0 == 0) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    float mmax = mj[q];
+#pragma unroll
+                    for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
+                    wj[q] = (lj[q] > 0.f) ? ex2(mj[q] - mmax) : 0.f;
+                    L[q] = wj[q] * lj[q];
+#pragma unroll
+                    for (int off = 16; off; off >>= 1) L[q] += __shfl_xor_sync(0xffffffffu, L[q], off);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const float w = (j0 + u < S) ? __shfl_sync(0xffffffffu, wj[q], min(j0 + u, 31)) : 0.f;
+                    // a partial without keys has weight 0 and its row was never written
+                    if (w != 0.f) {
+                        acc[q].x = fmaf(w, v[q][u].x, acc[q].x); acc[q].y = fmaf(w, v[q][u].y, acc[q].y);
+                        acc[q].z = fmaf(w, v[q][u].z, acc[q].z); acc[q].w = fmaf(w, v[q][u].w, acc[q].w);
+                    }
+                }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (s0 + q * n_warps < my_rows) store(rank + (s0 + q * n_warps) * S, acc[q], 1.f / L[q]);
+    }
+}
 
 // NSUB = 1: thread r of the softmax warps owns query row r and all 64 columns of a tile.
 // NSUB = 2 (units of at most 64 rows): the query rows are loaded twice, rows 64..127 being a
@@ -672,122 +766,74 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TM_COLS) : "memory");
     if (tid == 0 && *abort_flag && p.status) atomicOr(p.status, ORTHRUS_DEV_WAIT_TIMEOUT);
     if (S == 1 && NSUB == 1) return;
-    if (S > 1) cluster_sync_all();                            // every CTA's partial rows are in place
-
-    // Row R of the tile is merged and written by cluster rank R % S, which reads the row's S
-    // partial results out of its peers' shared memory: a warp per row, lane j holds the weight
-    // of the partial of rank j, every lane four output columns.  Rows are taken four at a time
-    // and all their loads are issued before the first is used, so that a warp pays the
-    // latency of the SM-to-SM path once per batch, not once per load.
-    const int my_rows = rank < rows_here ? (rows_here - rank + S - 1) / S : 0;
     constexpr int NWARPS = NTHREADS / 32;
-    if (my_rows <= NWARPS) {
-        // at most one row per warp: all of the row's partial results are requested at once
-        if (warp < my_rows) {
-            const int R = rank + warp * S;
-            float mj = -INFINITY, lj = 0.f;
-            if (lane < S) {
-                const uint32_t a = sbase + OFF_ML + R * 8;
-                const float2 v = ld_cluster_f2(S > 1 ? map_to_rank(a, lane) : a);
-                mj = v.x; lj = v.y;
-            }
-            const uint32_t a = sbase + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4);
-            float4 v[16];
-#pragma unroll
-            for (int u = 0; u < 16; ++u)
-                if (u < S) v[u] = ld_cluster_f4(S > 1 ? map_to_rank(a, u) : a);
-            float mmax = mj;
-#pragma unroll
-            for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
-            const float wj = (lj > 0.f) ? ex2(mj - mmax) : 0.f;
-            float L = wj * lj;
-#pragma unroll
-            for (int off = 16; off; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int u = 0; u < 16; ++u) {
-                const float w = (u < S) ? __shfl_sync(0xffffffffu, wj, u) : 0.f;
-                // a partial without keys has weight 0 and its row was never written
-                if (w != 0.f) {
-                    acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
-                    acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);
-                }
-            }
+    if (S == 1) {
+        // the two sub-streams of a lone CTA were folded in shared memory: normalise and write
+        const float *ml = reinterpret_cast<const float *>(smem + OFF_ML);
+        for (int R = warp; R < rows_here; R += NWARPS) {
+            const float4 v = *reinterpret_cast<const float4 *>(smem + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4));
+            const float inv = 1.f / ml[R * 2 + 1];
             const int i = i0 + R / p.G, g = R % p.G;
-            const float inv = 1.f / L;
             uint2 *dst = reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) +
                          (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD);
-            dst[lane] = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+            dst[lane] = make_uint2(pack_bf16(v.x * inv, v.y * inv), pack_bf16(v.z * inv, v.w * inv));
         }
-    } else
-    for (int s0 = warp; s0 < my_rows; s0 += 4 * NWARPS) {
-        float mj[4], lj[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int R = rank + min(s0 + q * NWARPS, my_rows - 1) * S;
-            mj[q] = -INFINITY; lj[q] = 0.f;
-            if (lane < S && s0 + q * NWARPS < my_rows) {
-                const uint32_t a = sbase + OFF_ML + R * 8;
-                const float2 v = ld_cluster_f2(S > 1 ? map_to_rank(a, lane) : a);
-                mj[q] = v.x; lj[q] = v.y;
-            }
-        }
-        float wj[4], L[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            float mmax = mj[q];
-#pragma unroll
-            for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
-            wj[q] = (lj[q] > 0.f) ? ex2(mj[q] - mmax) : 0.f;
-            L[q] = wj[q] * lj[q];
-#pragma unroll
-            for (int off = 16; off; off >>= 1) L[q] += __shfl_xor_sync(0xffffffffu, L[q], off);
-        }
-        float4 acc[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int j0 = 0; j0 < S; j0 += 4) {
-            float4 v[4][4];
+        return;
+    }
+
+    // How the CTAs of a cluster exchange their partial rows.  Up to 8 CTAs: each reads the
+    // rows it merges straight out of its peers' shared memory.  Larger clusters: through the
+    // workspace, which lives in L2 (an all-to-all of this size over the SM-to-SM path of a
+    // 16-CTA cluster moved about 5 bytes per cycle per SM and took longer than the whole
+    // stream of keys).  The cluster is what guarantees that the CTAs waiting for one another
+    // are resident together.
+    const int my_rows = rank < rows_here ? (rows_here - rank + S - 1) / S : 0;
+    auto store = [&](int R, const float4 &acc, float inv) {
+        const int i = i0 + R / p.G, g = R % p.G;
+        uint2 *dst = reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) +
+                     (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD);
+        dst[lane] = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+    };
+    if (S > kDsmemMaxCluster) {
+        const long long cta_lin = ((long long)rt * gridDim.y + order) * S + rank;
+        float *my_o = p.part_o + cta_lin * (MROWS * HD);
+        float *my_ml = p.part_ml + cta_lin * (MROWS * 2);
+        const float *ml = reinterpret_cast<const float *>(smem + OFF_ML);
+        // copy this CTA's rows out: a warp per row, 512 contiguous bytes
+        for (int R0 = warp; R0 < rows_here; R0 += 4 * NWARPS) {
+            float4 v[4];
+            float2 t2[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const int R = rank + min(s0 + q * NWARPS, my_rows - 1) * S;
-                const uint32_t a = sbase + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    // every CTA starts with its own partial, so that at any moment the CTAs of
-                    // the cluster read from different peers
-                    const int j = (min(j0 + u, S - 1) + rank) % S;
-                    if (s0 + q * NWARPS < my_rows) v[q][u] = ld_cluster_f4(S > 1 ? map_to_rank(a, j) : a);
-                }
+                const int R = min(R0 + q * NWARPS, rows_here - 1);
+                v[q] = *reinterpret_cast<const float4 *>(smem + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4));
+                t2[q] = *reinterpret_cast<const float2 *>(ml + R * 2);
             }
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int j = (min(j0 + u, S - 1) + rank) % S;
-                    const float w = (j0 + u < S) ? __shfl_sync(0xffffffffu, wj[q], j) : 0.f;
-                    // a partial without keys has weight 0 and its row was never written
-                    if (w != 0.f) {
-                        acc[q].x = fmaf(w, v[q][u].x, acc[q].x); acc[q].y = fmaf(w, v[q][u].y, acc[q].y);
-                        acc[q].z = fmaf(w, v[q][u].z, acc[q].z); acc[q].w = fmaf(w, v[q][u].w, acc[q].w);
-                    }
+            for (int q = 0; q < 4; ++q) {
+                const int R = R0 + q * NWARPS;
+                if (R < rows_here) {
+                    // (the row of a CTA without keys was never written: only its sum 0 matters)
+                    reinterpret_cast<float4 *>(my_o + R * HD)[lane] = v[q];
+                    if (lane == 0) *reinterpret_cast<float2 *>(my_ml + R * 2) = t2[q];
                 }
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int slot = s0 + q * NWARPS;
-            if (slot < my_rows) {
-                const int R = rank + slot * S;
-                const int i = i0 + R / p.G, g = R % p.G;
-                const float inv = 1.f / L[q];
-                uint2 *dst = reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) +
-                             (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD);
-                dst[lane] = make_uint2(pack_bf16(acc[q].x * inv, acc[q].y * inv),
-                                       pack_bf16(acc[q].z * inv, acc[q].w * inv));
             }
         }
+        cluster_sync_all();               // release / acquire at cluster scope: the rows are in place
+        const float *grp_o = p.part_o + (cta_lin - rank) * (MROWS * HD);
+        const float *grp_ml = p.part_ml + (cta_lin - rank) * (MROWS * 2);
+        merge_rows(S, rank, my_rows, warp, lane, NWARPS,
+                   [&](int j, int R) { return __ldcg(reinterpret_cast<const float2 *>(grp_ml + (long long)j * (MROWS * 2) + R * 2)); },
+                   [&](int j, int R) { return __ldcg(reinterpret_cast<const float4 *>(grp_o + (long long)j * (MROWS * HD) + R * HD) + lane); },
+                   store);
+        return;                           // nobody reads this CTA's shared memory
     }
-    if (S > 1) cluster_sync_all();     // peers may still be reading this CTA's rows
+    cluster_sync_all();                   // every CTA's partial rows are in place
+    merge_rows(S, rank, my_rows, warp, lane, NWARPS,
+               [&](int j, int R) { return ld_cluster_f2(map_to_rank(sbase + OFF_ML + R * 8, j)); },
+               [&](int j, int R) { return ld_cluster_f4(map_to_rank(sbase + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4), j)); },
+               store);
+    cluster_sync_all();                   // peers may still be reading this CTA's rows
 }
 
 // ---------------------------------------------------------------------------- host side
@@ -888,6 +934,7 @@ bool tc_path_supports(const AttnParams &p, int dtype)
 
 int tc_ctas_per_sm() { return 2; }
 int tc_tile_positions() { return TN; }
+int tc_dsmem_max_cluster() { return kDsmemMaxCluster; }
 
 template <int NSUB>
 static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int flags, cudaStream_t st)

@@ -58,6 +58,7 @@ cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st);  
 int tc_row_tiles(int G, int K);          // 128-row query tiles per unit (0: group too wide)
 int tc_ctas_per_sm();
 int tc_tile_positions();
+int tc_dsmem_max_cluster();             // larger clusters exchange split partials through the workspace
 cudaError_t launch_combine(const AttnParams &p, int dtype, cudaStream_t st);
 
 cudaError_t launch_consensus(const void *logits, int dtype, const int32_t *draft, int B, int K,

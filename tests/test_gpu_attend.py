@@ -78,7 +78,7 @@ def test_fp32_mode(view, shape):
 
 
 @pytest.mark.parametrize("view", VIEWS)
-@pytest.mark.parametrize("splits", [1, 2, 3, 7])
+@pytest.mark.parametrize("splits", [1, 2, 3, 7, 12, 16])
 @pytest.mark.parametrize("path", PATHS)
 def test_forced_splits_agree(view, splits, path):
     """Split-KV with empty, partial and full splits (ragged batch) gives the same result."""
