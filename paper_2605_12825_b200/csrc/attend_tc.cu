@@ -503,9 +503,15 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                     for (int q = 0; q < 4; ++q) m4[q] = fmaxf(m4[q], __uint_as_float(s[W - 4 + q]));
                     mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
                 } else {
+                    // a ragged or block tile: only the 16-column groups that hold visible keys
                     mx = -INFINITY;
 #pragma unroll
-                    for (int j = 0; j < W; ++j) if (j < lim) mx = fmaxf(mx, __uint_as_float(s[j]));
+                    for (int c = 0; c < W; c += 16) {
+                        if (c < lim) {
+#pragma unroll
+                            for (int j = c; j < c + 16; ++j) if (j < lim) mx = fmaxf(mx, __uint_as_float(s[j]));
+                        }
+                    }
                 }
                 const float m_new = fmaxf(m_run, mx * sc);
                 const bool need = m_new > m_run + RESCALE_THRESHOLD;   // also the first finite maximum
@@ -545,13 +551,21 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < W; j += 2) {
-                        float p0 = ex2(fmaf(__uint_as_float(s[j]), sc, neg_m));
-                        float p1 = ex2(fmaf(__uint_as_float(s[j + 1]), sc, neg_m));
-                        if (j >= lim) p0 = 0.f;
-                        if (j + 1 >= lim) p1 = 0.f;
-                        acc0.x += p0; acc0.y += p1;
-                        pk[j >> 1] = pack_bf16(p0, p1);
+                    for (int c = 0; c < W; c += 16) {
+                        if (c < lim) {
+#pragma unroll
+                            for (int j = c; j < c + 16; j += 2) {
+                                float p0 = ex2(fmaf(__uint_as_float(s[j]), sc, neg_m));
+                                float p1 = ex2(fmaf(__uint_as_float(s[j + 1]), sc, neg_m));
+                                if (j >= lim) p0 = 0.f;
+                                if (j + 1 >= lim) p1 = 0.f;
+                                acc0.x += p0; acc0.y += p1;
+                                pk[j >> 1] = pack_bf16(p0, p1);
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = c; j < c + 16; j += 2) pk[j >> 1] = 0u;
+                        }
                     }
                 }
                 l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
