@@ -46,6 +46,11 @@ def test_tiny_prefixes_bf16(view, P, path):
     (1, 32, 16, 2, 64, 333, 333),      # M = 256: two row tiles
     (2, 64, 2, 2, 128, 10, 90),        # widest block
     (1, 5, 6, 2, 64, 77, 77),          # M = 15, not a multiple of anything
+    (1, 64, 8, 2, 128, 150, 150),      # head_dim 128, M = 256: two row tiles of 32 positions
+    (2, 32, 16, 2, 128, 40, 500),      # G = 8, K = 32: M = 256, ragged
+    (1, 50, 6, 2, 128, 333, 333),      # G = 3: row tiles of 42 positions (126 rows), last one short
+    (1, 7, 20, 2, 128, 90, 90),        # G = 10: row tiles of 12 positions, K = 7 fits one
+    (2, 64, 64, 1, 128, 20, 200),      # G = 64: two positions per row tile, 32 row tiles
 ])
 @pytest.mark.parametrize("path", PATHS)
 def test_shapes_bf16(view, shape, path):
