@@ -147,27 +147,49 @@ class DeviceState:
         self.lens_host = W.prefix_lengths(wl)
         self.cache_len = self.lens_host.to(dev)
         self.cache_len0 = self.lens_host.to(dev)
-        self.host, self.t, self.layer, self.out_d, self.out_a = [], [], [], [], []
+        self.t, self.layer, self.out_d, self.out_a = [], [], [], []
         max_hint = int(self.lens_host.max())
+        lg = W.logits(wl)
+        greedy = lg.float().argmax(-1)          # input synthesis only: plants the agreement rate
+        draft = W.drafts(wl, greedy)
+        # Everything a step receives from the host (Q and block KV of both views for every
+        # layer, the AR logits, the drafts) lives in one pinned host arena and one device
+        # arena, so the end-to-end arm moves it with a single copy; the tensors the kernels
+        # see are 256-byte aligned views of the device arena.
+        host_layers = []
         for l in range(layers):
             h = W.attention_inputs(wl, layer=l)
             h.pop("cache_len")
-            t = {k: v.to(dev) for k, v in h.items()}
+            host_layers.append(h)
+        step_items = [(l, k, v) for l, h in enumerate(host_layers) for k, v in h.items() if "cache" not in k]
+        step_items += [(-1, "logits", lg), (-1, "draft", draft)]
+        offs, total = [], 0
+        for _, _, v in step_items:
+            offs.append(total)
+            total += (v.numel() * v.element_size() + 255) // 256 * 256
+        self.step_host = torch.empty(total, dtype=torch.uint8).pin_memory()
+        self.step_dev = torch.empty(total, dtype=torch.uint8, device=dev)
+        self.step_bytes_h2d = total
+        views = {}
+        for (l, k, v), off in zip(step_items, offs):
+            nb = v.numel() * v.element_size()
+            self.step_host[off:off + nb].view(v.dtype).view(v.shape).copy_(v)
+            views[(l, k)] = self.step_dev[off:off + nb].view(v.dtype).view(v.shape)
+        self.step_dev.copy_(self.step_host)
+        for l in range(layers):
+            h = host_layers[l]
+            t = {k: (v.to(dev) if "cache" in k else views[(l, k)]) for k, v in h.items()}
             self.t.append(t)
-            self.host.append({k: v.pin_memory() for k, v in h.items() if "cache" not in k})
             # in the step below no attention call directly follows a kernel that writes the
             # cache or its lengths, which is what the flag promises
             self.layer.append(B.make_layer(t["k_cache"], t["v_cache"], self.cache_len,
                                            wl.n_q_heads, wl.block, max_hint, 0.0, layer_flags))
             self.out_d.append(torch.empty_like(t["q_diff"]))
             self.out_a.append(torch.empty_like(t["q_ar"]))
+        del host_layers
+        self.logits = views[(-1, "logits")]
+        self.draft = views[(-1, "draft")]
         self.ws = B.new_workspace(B.orthrus_attend_workspace_bytes(self.layer[0]))
-        lg = W.logits(wl)
-        greedy = lg.float().argmax(-1)          # input synthesis only: plants the agreement rate
-        self.logits_host = lg.pin_memory()
-        self.draft_host = W.drafts(wl, greedy).pin_memory()
-        self.logits = lg.to(dev)
-        self.draft = self.draft_host.to(dev)
         Bn, K = wl.batch, wl.block
         i32 = dict(dtype=torch.int32, device=dev)
         self.n_commit = torch.zeros(Bn, **i32)
@@ -211,16 +233,9 @@ class DeviceState:
         return [self.phase_diffusion, self.phase_ar, self.phase_consensus, self.phase_commit]
 
     def h2d_inputs(self):
-        """End-to-end arm: this step's inputs come from pinned host memory."""
-        n = 0
-        for l in range(self.layers):
-            for k, hv in self.host[l].items():
-                self.t[l][k].copy_(hv, non_blocking=True)
-                n += hv.numel() * hv.element_size()
-        self.logits.copy_(self.logits_host, non_blocking=True)
-        self.draft.copy_(self.draft_host, non_blocking=True)
-        return n + self.logits_host.numel() * self.logits_host.element_size() + \
-            self.draft_host.numel() * 4
+        """End-to-end arm: this step's inputs come from pinned host memory, in one copy."""
+        self.step_dev.copy_(self.step_host, non_blocking=True)
+        return self.step_bytes_h2d
 
     def d2h_results(self):
         self.res_host.copy_(self.n_commit, non_blocking=True)
@@ -483,7 +498,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.CONFIGS))
