@@ -119,10 +119,17 @@ __device__ inline bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile in
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
 }
 
-__device__ inline void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, uint32_t bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
-                 " [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar) : "memory");
+// L2 policy for data that is read exactly once (the streamed cache tiles)
+__device__ inline uint64_t policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ inline void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, uint32_t bar,
+                                   uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+                 " [%0], [%1, {%2, %3}], [%4], %5;"
+                 ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar), "l"(policy) : "memory");
 }
 __device__ inline void tma_load_4d(uint32_t dst, const CUtensorMap *tm, int c0, int c1, int c2, int c3,
                                    uint32_t bar) {
@@ -432,6 +439,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     const int row_base = (int)(((long long)b * p.Hkv + h) * p.capacity);   // row of position 0
 
     // ring item j: tile j/2, K (even) or V (odd); slot j % NSLOT
+    const uint64_t stream_policy = policy_evict_first();
     auto issue_item = [&](int j) {
         const int t = j >> 1, slot = j % NSLOT;
         const bool is_v = j & 1;
@@ -441,8 +449,8 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
         if (t < n_mine) {
             const CUtensorMap *m = is_v ? &tm.v : &tm.k;
             const int row = row_base + ((int)t0 + t) * TN;
-            tma_load_2d(dst, m, 0, row, fb);
-            tma_load_2d(dst + SUB_BYTES, m, 64, row, fb);
+            tma_load_2d(dst, m, 0, row, fb, stream_policy);
+            tma_load_2d(dst + SUB_BYTES, m, 64, row, fb, stream_policy);
         } else {                  // block tile: rows >= K are out of bounds and arrive as zeros
             const CUtensorMap *m = is_v ? &tm.vb : &tm.kb;
             tma_load_4d(dst, m, 0, h, 0, b, fb);
