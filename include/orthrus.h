@@ -105,7 +105,9 @@ enum {
  * Bytes of workspace the two attention calls (and orthrus_kv_append) need for
  * this layer shape: a 256-byte header holding the status word, followed by the
  * split-KV partial results (written and read back inside one call; they are meant
- * to stay in L2).  Returns 0 for an invalid descriptor.
+ * to stay in L2).  A workspace serves one stream at a time: calls on the same stream
+ * may share it, calls that can overlap on the GPU (different streams) need their own.
+ * Returns 0 for an invalid descriptor.
  */
 size_t orthrus_attend_workspace_bytes(const orthrus_layer_t *layer);
 
