@@ -103,7 +103,8 @@ static Plan make_plan(const orthrus_layer_t *L, bool tc)
             //  still split; many small CTAs would spend their time starting and merging)
             while (S < 16 && units * S < slots && tiles / (S * 2) >= 8) S *= 2;
         }
-        if (S > 16) S = 16;
+        const int max_cluster = tc_max_cluster();
+        if (S > max_cluster) S = max_cluster;
         if (S > tiles) S = tiles;
         if (S < 1) S = 1;
         pl.n_splits = S;

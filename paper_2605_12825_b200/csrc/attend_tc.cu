@@ -955,6 +955,42 @@ bool tc_path_supports(const AttnParams &p, int dtype)
 }
 
 int tc_ctas_per_sm() { return 2; }
+
+// Largest cluster size (a power of two up to 16) the current device can co-schedule for this
+// kernel; 16 on a full B200.  Without a device (or if the query fails) 16 is assumed and a
+// launch that cannot be scheduled reports its error.
+int tc_max_cluster()
+{
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static int cached[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 16;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[dev]) return cached[dev];
+    int best = 16;
+    if (cudaFuncSetAttribute(attend_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(attend_tc_kernel<1>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+        for (int s = 16; s >= 2; s >>= 1) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(s, 1, 1);
+            cfg.blockDim = dim3(NTHREADS);
+            cfg.dynamicSmemBytes = SMEM_BYTES;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = s; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, attend_tc_kernel<1>, &cfg) == cudaSuccess && n > 0) { best = s; break; }
+            best = s >> 1;
+        }
+        if (best < 1) best = 1;
+    } else {
+        (void)cudaGetLastError();
+    }
+    cached[dev] = best;
+    return best;
+}
 int tc_tile_positions() { return TN; }
 int tc_dsmem_max_cluster() { return kDsmemMaxCluster; }
 
@@ -962,14 +998,23 @@ template <int NSUB>
 static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int flags, cudaStream_t st)
 {
     const int S = p.n_splits;
-    static std::once_flag once;
-    static cudaError_t cfg_err = cudaSuccess;
-    std::call_once(once, [] {
-        cfg_err = cudaFuncSetAttribute(attend_tc_kernel<NSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-        if (cfg_err == cudaSuccess)
-            cfg_err = cudaFuncSetAttribute(attend_tc_kernel<NSUB>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-    });
-    if (cfg_err != cudaSuccess) return cfg_err;
+    {   // function attributes belong to a device: set them once on each device that launches
+        constexpr int kMaxDevices = 64;
+        static std::mutex mu;
+        static bool configured[kMaxDevices] = {};
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> lock(mu);
+        if (!configured[dev]) {
+            e = cudaFuncSetAttribute(attend_tc_kernel<NSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(attend_tc_kernel<NSUB>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            if (e != cudaSuccess) return e;
+            configured[dev] = true;
+        }
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(S, p.B * p.Hkv, (p.K + kb - 1) / kb);
     cfg.blockDim = dim3(NTHREADS);

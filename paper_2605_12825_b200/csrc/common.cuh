@@ -57,6 +57,7 @@ bool tc_path_supports(const AttnParams &p, int dtype);
 cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st);   // n_splits = cluster size
 int tc_row_tiles(int G, int K);          // 128-row query tiles per unit (0: group too wide)
 int tc_ctas_per_sm();
+int tc_max_cluster();                   // largest cluster the device can co-schedule (<= 16)
 int tc_tile_positions();
 int tc_dsmem_max_cluster();             // larger clusters exchange split partials through the workspace
 cudaError_t launch_combine(const AttnParams &p, int dtype, cudaStream_t st);
