@@ -28,12 +28,12 @@
 //
 // Merge.  Every softmax thread puts its partial row (max, sum, unnormalised O straight out
 // of TMEM) into its CTA's idle ring.  Row r of the tile is merged and written by cluster
-// rank r % S.  Clusters of up to 8 CTAs read the rows they merge straight out of their
-// peers' shared memory, between two cluster barriers.  Larger clusters go through the
+// rank r % S.  Small exchanges (cluster size x rows < 1024) are read straight out of the
+// peers' shared memory, between two cluster barriers.  Larger ones go through the
 // workspace (L2): each CTA copies its rows out with 512-byte coalesced stores, one cluster
 // barrier publishes them, the owners read them back and a CTA leaves as soon as its own
-// rows are written; for a 16-CTA all-to-all the SM-to-SM path was measured to be slower
-// than that.  There is no second kernel.
+// rows are written; for those sizes the SM-to-SM path was measured to be slower.  There is
+// no second kernel.
 //
 // Programmatic dependent launch.  The kernel waits for the preceding kernel of the
 // stream (griddepcontrol.wait) before it reads anything that kernel may have written,
@@ -79,7 +79,9 @@ static_assert(NUM_BARS <= 24, "barrier area");
 
 constexpr uint32_t TM_O = 0, TM_S = 128, TM_COLS = 256;   // TMEM column map
 constexpr float RESCALE_THRESHOLD = 8.f;                  // log2 units
-constexpr int kDsmemMaxCluster = 8;                       // larger clusters exchange partials through L2
+// a cluster whose partial rows add up to this many (cluster size x rows per CTA) or more
+// exchanges them through the L2 workspace instead of distributed shared memory
+constexpr int kL2ExchangeRows = 1024;
 
 __device__ inline uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -803,12 +805,12 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
         return;
     }
 
-    // How the CTAs of a cluster exchange their partial rows.  Up to 8 CTAs: each reads the
-    // rows it merges straight out of its peers' shared memory.  Larger clusters: through the
-    // workspace, which lives in L2 (an all-to-all of this size over the SM-to-SM path of a
-    // 16-CTA cluster moved about 5 bytes per cycle per SM and took longer than the whole
-    // stream of keys).  The cluster is what guarantees that the CTAs waiting for one another
-    // are resident together.
+    // How the CTAs of a cluster exchange their partial rows.  Small exchanges: each CTA reads
+    // the rows it merges straight out of its peers' shared memory.  Large ones (cluster size x
+    // rows >= 1024, e.g. 16 CTAs x 64 rows or 8 x 128): through the workspace, which lives in
+    // L2; an all-to-all of that size over the SM-to-SM path moved about 5 bytes per cycle per
+    // SM and took longer than the whole stream of keys.  The cluster is what guarantees that
+    // the CTAs waiting for one another are resident together.
     const int my_rows = rank < rows_here ? (rows_here - rank + S - 1) / S : 0;
     auto store = [&](int R, const float4 &acc, float inv) {
         const int i = i0 + R / p.G, g = R % p.G;
@@ -816,7 +818,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                      (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD);
         dst[lane] = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
     };
-    if (S > kDsmemMaxCluster) {
+    if (S * rows_here >= kL2ExchangeRows) {
         const long long cta_lin = ((long long)rt * gridDim.y + order) * S + rank;
         float *my_o = p.part_o + cta_lin * (MROWS * HD);
         float *my_ml = p.part_ml + cta_lin * (MROWS * 2);
@@ -992,7 +994,7 @@ int tc_max_cluster()
     return best;
 }
 int tc_tile_positions() { return TN; }
-int tc_dsmem_max_cluster() { return kDsmemMaxCluster; }
+bool tc_exchange_in_workspace(int S, int M) { return S * (M < MROWS ? M : MROWS) >= kL2ExchangeRows; }
 
 template <int NSUB>
 static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int flags, cudaStream_t st)
