@@ -13,7 +13,8 @@
 //              the bf16 probabilities back into TMEM over the scores, where the P.V
 //              product reads them as its A operand.
 //   warp 4     producer: one lane issues every TMA load (Q tile, K and V tiles of the
-//              cache, the block K/V tile) into a ring of five 16 KB slots.
+//              cache, the block K/V tile) into a ring of five 16 KB slots, in the order
+//              the MMAs consume them.
 //   warp 5     TMEM allocation and MMA issue: S = Q.K^T into one of two score buffers
 //              (so that QK(t+1) runs under softmax(t)), then O += P.V.
 // The output accumulator O stays in TMEM for the whole CTA.  The running max is only
@@ -440,11 +441,17 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     const bool active = n_tiles > 0 && aligned;
     const int row_base = (int)(((long long)b * p.Hkv + h) * p.capacity);   // row of position 0
 
-    // ring item j: tile j/2, K (even) or V (odd); slot j % NSLOT
+    // The ring holds K and V tiles in the order the MMAs consume them: K0, K1, V0, K2, V1, ...,
+    // K(n-1), V(n-2), V(n-1) (the product P.V of a tile is issued after the scores of the next
+    // one), so that slots are freed in the order they were filled and a V tile does not sit
+    // in the ring while its softmax is still to come.  Item j lives in slot j % NSLOT.
+    auto item_of_k = [&](int t) { return t == 0 ? 0 : 2 * t - 1; };
+    auto item_of_v = [&](int t) { return min(2 * t + 2, 2 * n_tiles - 1); };
     const uint64_t stream_policy = policy_evict_first();
     auto issue_item = [&](int j) {
-        const int t = j >> 1, slot = j % NSLOT;
-        const bool is_v = j & 1;
+        const int slot = j % NSLOT;
+        const bool is_v = j == 2 * n_tiles - 1 || (j > 0 && (j & 1) == 0);
+        const int t = is_v ? (j == 2 * n_tiles - 1 ? n_tiles - 1 : j / 2 - 1) : (j + 1) / 2;
         const uint32_t dst = sbase + OFF_RING + slot * SLOT_BYTES;
         const uint32_t fb = bar(BAR_FULL + slot);
         mbar_expect_tx(fb, SLOT_BYTES);
@@ -464,7 +471,9 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
         // the cache rows below cache_len are not being written by the preceding kernel:
         // request the first prefix tiles before waiting for it
         if (active && warp == 4 && lane == 0)
-            while (produced < 2 * n_mine && produced < NSLOT) { issue_item(produced); ++produced; }
+            while (produced < (owner ? item_of_k(n_tiles - 1) : 2 * n_tiles) && produced < NSLOT) {
+                issue_item(produced); ++produced;     // (stops before the block tile's first item)
+            }
         griddep_wait();
     }
     griddep_launch();
@@ -723,7 +732,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
         constexpr uint32_t IDESC_QK = make_idesc(TN, 0);      // A = Q, B = K tile, both K-major
         constexpr uint32_t IDESC_PV = make_idesc(HD, 1);      // A = P (TMEM), B = V tile (MN-major)
         auto issue_qk = [&](int t) -> bool {
-            const int j = 2 * t, slot = j % NSLOT;
+            const int j = item_of_k(t), slot = j % NSLOT;
             if (!mbar_wait_warp(bar(BAR_FULL + slot), (j / NSLOT) & 1, abort_flag)) return false;
             tc_fence_after();
             if (lane == 0) {
@@ -742,7 +751,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             return true;
         };
         auto issue_pv = [&](int t) -> bool {
-            const int j = 2 * t + 1, slot = j % NSLOT;
+            const int j = item_of_v(t), slot = j % NSLOT;
             if (!mbar_wait_warp(bar(BAR_FULL + slot), (j / NSLOT) & 1, abort_flag)) return false;
             // a ragged prefix tile: V rows past the prefix may hold anything, and 0 * NaN would
             // poison the product, so they are cleared before the MMA reads them
