@@ -50,7 +50,7 @@ def measured_peak():
 # DRAM bytes (read + write) per launch of the attention kernel from the ncu capture summarised
 # in profiles/attend_tc_cfg2_8b_b1.md, with the first 16 hex digits of the SHA-256 of the
 # kernel source the capture was taken from: once that file changes the figure is stale.
-NCU_TRAFFIC = {"cfg2_8b_b1": (17045760, "5022ee0e01cd465d")}
+NCU_TRAFFIC = {"cfg2_8b_b1": (17048320, "5022ee0e01cd465d")}
 
 
 def recorded_traffic(workload: str):
