@@ -194,6 +194,12 @@ class DeviceState:
             # cache or its lengths, which is what the flag promises
             self.layer.append(B.make_layer(t["k_cache"], t["v_cache"], self.cache_len,
                                            wl.n_q_heads, wl.block, max_hint, 0.0, layer_flags))
+            if l == 0:
+                # the step's first attention call follows the kernel that rewinds cache_len (an
+                # artefact of replaying the same step): no promise is made for that one call
+                self.layer0_first = B.make_layer(t["k_cache"], t["v_cache"], self.cache_len, wl.n_q_heads,
+                                                 wl.block, max_hint, 0.0,
+                                                 layer_flags & ~B.LAYER_CACHE_QUIESCENT)
             self.out_d.append(torch.empty_like(t["q_diff"]))
             self.out_a.append(torch.empty_like(t["q_ar"]))
         del host_layers
@@ -216,8 +222,8 @@ class DeviceState:
         B = self.B
         for l in range(self.layers):
             t = self.t[l]
-            B.orthrus_diffusion_block_attend(self.layer[l], t["q_diff"], t["k_diff_blk"],
-                                             t["v_diff_blk"], self.out_d[l], self.ws)
+            B.orthrus_diffusion_block_attend(self.layer0_first if l == 0 else self.layer[l], t["q_diff"],
+                                             t["k_diff_blk"], t["v_diff_blk"], self.out_d[l], self.ws)
 
     def phase_ar(self):
         B = self.B

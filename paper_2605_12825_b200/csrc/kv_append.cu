@@ -32,34 +32,34 @@ __global__ void __launch_bounds__(256) kv_append_kernel(
     if (update_len && threadIdx.x == 0) cache_len[b] = P + n;
 }
 
-// Several layers in one launch.  CTA (b, l) copies layer l's accepted rows of sequence b;
-// the lengths are left alone, so every CTA sees the same P_b whatever the order they run in.
+// Several layers in one launch.  CTA (b, l, h) copies the accepted rows of KV head h of layer
+// l of sequence b; the lengths are left alone, so every CTA sees the same P_b whatever the
+// order they run in.
 constexpr int kLayersPerLaunch = 64;
 struct AppendBatch { AppendLayer layer[kLayersPerLaunch]; };
 
-__global__ void __launch_bounds__(256) kv_append_layers_kernel(
+__global__ void __launch_bounds__(128) kv_append_layers_kernel(
     const __grid_constant__ AppendBatch batch, const int32_t *n_commit, int K, int Hkv, int row_vecs,
     long long capacity, int32_t *status)
 {
-    const int b = blockIdx.x;
+    const int b = blockIdx.x, h = blockIdx.z;
     const AppendLayer &L = batch.layer[blockIdx.y];
     const int P = L.cache_len[b];
     const int n = n_commit[b];
     if (n < 0 || n > K || P < 0 || (long long)P + n > capacity) {
-        if (status && threadIdx.x == 0) atomicOr(status, ORTHRUS_DEV_APPEND_OVERFLOW);
+        if (status && threadIdx.x == 0 && h == 0) atomicOr(status, ORTHRUS_DEV_APPEND_OVERFLOW);
         return;
     }
     uint4 *kc = static_cast<uint4 *>(L.k_cache), *vc = static_cast<uint4 *>(L.v_cache);
     const uint4 *kb = static_cast<const uint4 *>(L.k_blk), *vb = static_cast<const uint4 *>(L.v_blk);
-    const int total = n * Hkv * row_vecs;
+    // the n destination rows of this head are contiguous: [P, P + n) x row_vecs vectors
+    const long long dst0 = (((long long)b * Hkv + h) * capacity + P) * row_vecs;
+    const int total = n * row_vecs;
     for (int e = threadIdx.x; e < total; e += blockDim.x) {
-        const int c = e % row_vecs;
-        const int h = (e / row_vecs) % Hkv;
-        const int i = e / (row_vecs * Hkv);
+        const int i = e / row_vecs, c = e - i * row_vecs;
         const long long src = (((long long)b * K + i) * Hkv + h) * row_vecs + c;
-        const long long dst = (((long long)b * Hkv + h) * capacity + P + i) * row_vecs + c;
-        kc[dst] = kb[src];
-        vc[dst] = vb[src];
+        kc[dst0 + e] = kb[src];
+        vc[dst0 + e] = vb[src];
     }
 }
 
@@ -91,7 +91,7 @@ cudaError_t launch_kv_append_layers(const orthrus_layer_t &shape, const AppendLa
         const int n = n_layers - l0 < kLayersPerLaunch ? n_layers - l0 : kLayersPerLaunch;
         for (int l = 0; l < n; ++l) batch.layer[l] = layers[l0 + l];
         for (int l = n; l < kLayersPerLaunch; ++l) batch.layer[l] = layers[l0];
-        kv_append_layers_kernel<<<dim3(shape.batch, n), 256, 0, st>>>(
+        kv_append_layers_kernel<<<dim3(shape.batch, n, shape.n_kv_heads), 128, 0, st>>>(
             batch, n_commit, shape.block, shape.n_kv_heads, row_vecs, shape.capacity, status);
         count_launch();
         cudaError_t e = cudaGetLastError();
@@ -101,8 +101,9 @@ cudaError_t launch_kv_append_layers(const orthrus_layer_t &shape, const AppendLa
         LenBatch lb;
         for (int j = 0; j < 128; ++j) lb.len[j] = len_arrays[j < n_len_arrays ? j : 0];
         const int total = shape.batch * n_len_arrays;
-        kv_append_bump_kernel<<<(total + 255) / 256 < 64 ? (total + 255) / 256 : 64, 256, 0, st>>>(
-            lb, n_len_arrays, n_commit, shape.batch, shape.block, shape.capacity);
+        const int blocks = (total + 255) / 256 < 64 ? (total + 255) / 256 : 64;
+        kv_append_bump_kernel<<<blocks, 256, 0, st>>>(lb, n_len_arrays, n_commit, shape.batch, shape.block,
+                                                      shape.capacity);
         count_launch();
         return cudaGetLastError();
     }
