@@ -415,7 +415,7 @@ def run_gpu(args):
     }
     if rank == 0:
         if not args.no_cpu_baseline and world == 1:
-            out["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_budget)
+            out["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_budget, gpu_state=st)
         print(json.dumps(out), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -439,16 +439,19 @@ def oracle_sample(wl: W.Workload, layer: int = 0):
     return t, rows, lg
 
 
-def oracle_step(wl, t, rows, lg):
+def oracle_step(wl, t, rows, lg, draft=None):
+    """One bounded sample of the path on the CPU oracle; returns what it computed."""
     import oracle
-    oracle.block_attend_rows(oracle.VIEW_DIFFUSION, rows, t["q_diff"], t["k_diff_blk"],
-                             t["v_diff_blk"], t["k_cache"], t["v_cache"], t["cache_len"])
-    oracle.block_attend_rows(oracle.VIEW_AR, rows, t["q_ar"], t["k_ar_blk"], t["v_ar_blk"],
-                             t["k_cache"], t["v_cache"], t["cache_len"])
-    draft = torch.zeros(wl.batch, wl.block, dtype=torch.int32)
-    n, *_ = oracle.consensus_accept(lg, draft)
+    od = oracle.block_attend_rows(oracle.VIEW_DIFFUSION, rows, t["q_diff"], t["k_diff_blk"],
+                                  t["v_diff_blk"], t["k_cache"], t["v_cache"], t["cache_len"])
+    oa = oracle.block_attend_rows(oracle.VIEW_AR, rows, t["q_ar"], t["k_ar_blk"], t["v_ar_blk"],
+                                  t["k_cache"], t["v_cache"], t["cache_len"])
+    if draft is None:
+        draft = torch.zeros(wl.batch, wl.block, dtype=torch.int32)
+    cons = oracle.consensus_accept(lg, draft)
     lens = t["cache_len"].clone()
-    oracle.kv_append(t["k_cache"], t["v_cache"], lens, t["k_ar_blk"], t["v_ar_blk"], n)
+    oracle.kv_append(t["k_cache"], t["v_cache"], lens, t["k_ar_blk"], t["v_ar_blk"], cons[0])
+    return od, oa, cons
 
 
 def sample_bytes(wl, t, rows):
@@ -459,27 +462,49 @@ def sample_bytes(wl, t, rows):
     return full * rows.shape[0] / (wl.batch * wl.block * wl.n_q_heads)
 
 
-def cpu_baseline(wl, budget_s=20.0):
+def cpu_baseline(wl, budget_s=20.0, gpu_state=None):
     """Times the oracle, as it stands, on samples of successive layers until about
-    `budget_s` core-seconds of CPU work have been spent."""
+    `budget_s` core-seconds of CPU work have been spent.  With `gpu_state` (the device
+    tensors the timed region left behind) the rows the oracle has just computed are also
+    compared with the GPU's outputs of the last timed step, so the timed kernels are known
+    to have produced the real results."""
     import oracle
     oracle.build()
     cores = oracle.num_threads()
     spent, nbytes, layer, rows_n = 0.0, 0.0, 0, 0
     lg = W.logits(wl)
+    draft = gpu_state.draft.cpu() if gpu_state is not None else None
+    worst, checked = 0.0, 0
     while spent * cores < budget_s and layer < max(wl.layers, 8):
         t, rows, _ = oracle_sample(wl, layer)
         t0 = time.perf_counter()
-        oracle_step(wl, t, rows, lg)
+        od, oa, cons = oracle_step(wl, t, rows, lg, draft)
         spent += time.perf_counter() - t0
         nbytes += sample_bytes(wl, t, rows)
         rows_n = rows.shape[0]
+        if gpu_state is not None and layer < gpu_state.layers:
+            idx = (rows[:, 0].long(), rows[:, 1].long(), rows[:, 2].long())
+            for ref, out in ((od, gpu_state.out_d[layer]), (oa, gpu_state.out_a[layer])):
+                err = float((out.cpu().double()[idx] - ref).abs().max())
+                scale = float(ref.abs().max())
+                if not (err <= 2e-2 and err <= 1e-2 * scale):
+                    raise SystemExit(f"bench.py: layer {layer}: attention output of the timed step is off "
+                                     f"the oracle (max-abs {err:.3e}, max|ref| {scale:.3e})")
+                worst = max(worst, err / scale)
+                checked += rows.shape[0]
+            if layer == 0 and not (torch.equal(gpu_state.n_commit.cpu(), cons[0]) and
+                                   torch.equal(gpu_state.committed.cpu(), cons[1])):
+                raise SystemExit("bench.py: consensus of the timed step differs from the oracle")
         layer += 1
-    return {"value": round(nbytes / spent / 1e9, 4), "unit": "GB/s", "cores": cores,
-            "kind": "oracle", "seconds": round(spent, 3),
-            "sample": f"{wl.name}: {layer} layer(s), both views, {rows_n} of "
-                      f"{wl.batch * wl.block * wl.n_q_heads} query rows per layer, each with a "
-                      f"full consensus and commit"}
+    out = {"value": round(nbytes / spent / 1e9, 4), "unit": "GB/s", "cores": cores,
+           "kind": "oracle", "seconds": round(spent, 3),
+           "sample": f"{wl.name}: {layer} layer(s), both views, {rows_n} of "
+                     f"{wl.batch * wl.block * wl.n_q_heads} query rows per layer, each with a "
+                     f"full consensus and commit"}
+    if gpu_state is not None:
+        out["gpu_outputs_checked"] = {"attention_rows": checked, "max_err_over_max_ref": round(worst, 5),
+                                      "consensus": "bit-exact"}
+    return out
 
 
 def run_reference(args):
