@@ -288,6 +288,8 @@ def run_gpu(args):
     from paper_2605_12825_b200 import binding as B
 
     wl = W.CONFIGS[args.workload]
+    if args.block:
+        wl = wl.with_(block=args.block, name=f"{wl.name}_K{args.block}")
     layers = args.layers or wl.layers
     flags = 0 if args.no_early_prefetch else B.LAYER_CACHE_QUIESCENT
     if args.no_early_launch:
@@ -544,6 +546,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.CONFIGS))
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count")
+    ap.add_argument("--block", type=int, default=0,
+                    help="override the block width K (the block-size sweep of Section 5)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-early-prefetch", action="store_true",
                     help="do not set ORTHRUS_LAYER_CACHE_QUIESCENT on the layers")
