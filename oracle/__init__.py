@@ -67,6 +67,12 @@ def lib() -> ctypes.CDLL:
                                                  ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                                  ctypes.c_void_p, ctypes.c_void_p,
                                                  ctypes.c_void_p, ctypes.c_void_p]
+        _lib.oracle_consensus_sample.restype = ctypes.c_int
+        _lib.oracle_consensus_sample.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                                                 ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                                 ctypes.c_double, ctypes.c_int32, ctypes.c_int32,
+                                                 ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                                 ctypes.c_void_p, ctypes.c_void_p]
         _lib.oracle_kv_append.restype = ctypes.c_int
         _lib.oracle_kv_append.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                           ctypes.c_int32, ctypes.c_int64, ctypes.c_int,
@@ -162,6 +168,35 @@ def consensus_accept(logits: torch.Tensor, draft: torch.Tensor
     if rc != 0:
         raise RuntimeError(f"oracle_consensus_accept failed ({rc})")
     return n, com, arg, nxt
+
+
+def consensus_sample(ar_logits: torch.Tensor, diff_logits: torch.Tensor, draft: torch.Tensor,
+                     u_accept: torch.Tensor, u_resample: torch.Tensor, temperature: float):
+    """Sampled consensus for T > 0 (the rejection-sampling rule of Section 3.3).
+    u_accept, u_resample: [B][K] in [0, 1).  Returns (n_commit [B], committed [B][K],
+    next_anchor [B]) int32 and margin [B] float64 (distance of the nearest decision
+    from flipping, relative)."""
+    _check(ar_logits, "ar_logits")
+    _check(diff_logits, "diff_logits")
+    _check(draft, "draft")
+    B, K, V = ar_logits.shape
+    if diff_logits.shape != ar_logits.shape or diff_logits.dtype != ar_logits.dtype:
+        raise ValueError("the two logit tensors must agree in shape and dtype")
+    if draft.dtype != torch.int32 or tuple(draft.shape) != (B, K):
+        raise ValueError("draft must be int32 [B][K]")
+    ua = u_accept.to(torch.float64).contiguous()
+    ur = u_resample.to(torch.float64).contiguous()
+    n = torch.empty(B, dtype=torch.int32)
+    com = torch.empty((B, K), dtype=torch.int32)
+    nxt = torch.empty(B, dtype=torch.int32)
+    margin = torch.empty(B, dtype=torch.float64)
+    rc = lib().oracle_consensus_sample(ar_logits.data_ptr(), diff_logits.data_ptr(),
+                                       _DTYPE_CODE[ar_logits.dtype], draft.data_ptr(),
+                                       ua.data_ptr(), ur.data_ptr(), float(temperature), B, K, V,
+                                       n.data_ptr(), com.data_ptr(), nxt.data_ptr(), margin.data_ptr())
+    if rc != 0:
+        raise RuntimeError(f"oracle_consensus_sample failed ({rc})")
+    return n, com, nxt, margin
 
 
 def kv_append(k_cache, v_cache, cache_len, k_blk, v_blk, n_commit, update_len: bool = True) -> int:

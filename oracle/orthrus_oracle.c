@@ -17,10 +17,13 @@
  *   cache_len     [B] int32   (P_b = number of valid prefix positions)
  *   logits        [B][K][V];  draft, committed, ar_argmax [B][K] int32
  *
- * Parity status: every function here is pinned by tests/test_oracle_pins.py
- * (brute-force mask-matrix softmax, closed forms, K=1 reduction, permutation
- * invariances, sequential greedy decoding of a toy model, byte-level append
- * checks).  Nothing is "parity unpinned".
+ * Parity status: every function here is pinned by tests/test_oracle_pins.py and
+ * tests/test_oracle_sampling_pins.py (brute-force mask-matrix softmax, closed forms,
+ * K=1 reduction, permutation invariances, sequential greedy decoding of a toy
+ * model, byte-level append checks; for the sampled consensus: the committed token
+ * follows the AR distribution, acceptance rate 1 - total variation, reduction to
+ * the greedy rule at low temperature, library inverse-CDF on the degenerate
+ * cases).  Nothing is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -231,6 +234,119 @@ int oracle_consensus_accept(const void *logits, int dtype, const int32_t *draft,
         next_anchor[b] = g[n - 1];
     }
     return 0;
+}
+
+/*
+ * Sampled consensus for temperature T > 0 (Section 3.3: "exact rejection sampling",
+ * the speculative-sampling rule of the work it cites, which keeps the committed
+ * tokens distributed exactly as the AR view would have sampled them).
+ *
+ * With p_k = softmax(ar_logits[b][k] / T) and q_k = softmax(diff_logits[b][k] / T),
+ * the drafts are visited left to right.  Draft y_k (drawn from q_k by the caller) is
+ * kept iff  u_accept[b][k] * q_k(y_k) <= p_k(y_k),  i.e. with probability
+ * min(1, p_k(y_k) / q_k(y_k)).  At the first k that fails, verification halts and the
+ * correction token is drawn from the residual distribution
+ *     r(v) = max(0, p_k(v) - q_k(v)) / sum_w max(0, p_k(w) - q_k(w))
+ * by inverting its running sum with u_resample[b][k]: the smallest v whose running
+ * sum exceeds u * total.  (If the residual is identically zero, which exact
+ * arithmetic allows only when nothing can be rejected, p_k itself is inverted.)
+ * n = kept drafts + 1 correction token, or K when every draft is kept (there is no
+ * further verified row: the same reading as in the greedy rule).
+ *
+ * u_accept, u_resample: [B][K] doubles in [0, 1), supplied by the caller.
+ * Outputs: n_commit [B], committed [B][K] (-1 beyond n), next_anchor [B], and
+ * margin [B] (optional): how far the nearest decision of sequence b was from
+ * flipping, relative to the quantities compared (min over the accept tests taken
+ * of |u*q(y) - p(y)| / max(p(y), u*q(y)) and, if a token was resampled, of the
+ * distance of u*total to the two running sums that bracket it, over total).
+ */
+int oracle_consensus_sample(const void *ar_logits, const void *diff_logits, int dtype,
+                            const int32_t *draft, const double *u_accept,
+                            const double *u_resample, double temperature,
+                            int32_t B, int32_t K, int32_t V,
+                            int32_t *n_commit, int32_t *committed, int32_t *next_anchor,
+                            double *margin)
+{
+    if (B < 0 || K <= 0 || V <= 0 || !(temperature > 0.0)) return -2;
+    int rc = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t b = 0; b < B; ++b) {
+        double *p = (double *)malloc(sizeof(double) * (size_t)V);
+        double *q = (double *)malloc(sizeof(double) * (size_t)V);
+        if (!p || !q) {
+            free(p); free(q);
+#pragma omp atomic write
+            rc = -1;
+            continue;
+        }
+        double worst = INFINITY;
+        int32_t n = 0;
+        for (int32_t k = 0; k < K; ++k) {
+            const int64_t row = ((int64_t)b * K + k) * V;
+            double mp = -INFINITY, mq = -INFINITY;
+            for (int32_t v = 0; v < V; ++v) {
+                p[v] = load_elem(ar_logits, dtype, row + v) / temperature;
+                q[v] = load_elem(diff_logits, dtype, row + v) / temperature;
+                if (p[v] > mp) mp = p[v];
+                if (q[v] > mq) mq = q[v];
+            }
+            double zp = 0.0, zq = 0.0;
+            for (int32_t v = 0; v < V; ++v) {
+                p[v] = exp(p[v] - mp); zp += p[v];
+                q[v] = exp(q[v] - mq); zq += q[v];
+            }
+            for (int32_t v = 0; v < V; ++v) { p[v] /= zp; q[v] /= zq; }
+
+            const int32_t y = draft[(int64_t)b * K + k];
+            const double lhs = u_accept[(int64_t)b * K + k] * q[y], rhs = p[y];
+            const double big = lhs > rhs ? lhs : rhs;
+            const double m1 = big > 0.0 ? fabs(lhs - rhs) / big : INFINITY;
+            if (m1 < worst) worst = m1;
+            if (lhs <= rhs) {                       /* draft kept */
+                committed[(int64_t)b * K + n] = y;
+                ++n;
+                continue;
+            }
+            /* first rejection: draw the correction token from the residual */
+            double total = 0.0;
+            for (int32_t v = 0; v < V; ++v) { const double r = p[v] - q[v]; if (r > 0.0) total += r; }
+            const int use_p = !(total > 0.0);
+            if (use_p) total = 1.0;
+            const double target = u_resample[(int64_t)b * K + k] * total;
+            double run = 0.0, prev = 0.0;
+            int32_t z = -1;
+            for (int32_t v = 0; v < V; ++v) {
+                const double r = use_p ? p[v] : (p[v] - q[v] > 0.0 ? p[v] - q[v] : 0.0);
+                if (r > 0.0) {
+                    prev = run;
+                    run += r;
+                    if (run > target) { z = v; break; }
+                }
+            }
+            if (z < 0) {                            /* rounding left the last sum at or below target */
+                for (int32_t v = V - 1; v >= 0; --v) {
+                    const double r = use_p ? p[v] : p[v] - q[v];
+                    if (r > 0.0) { z = v; break; }
+                }
+                if (z < 0) z = 0;
+                prev = run;
+            }
+            {
+                const double lo = fabs(target - prev) / total, hi = fabs(run - target) / total;
+                const double m2 = lo < hi ? lo : hi;
+                if (m2 < worst) worst = m2;
+            }
+            committed[(int64_t)b * K + n] = z;
+            ++n;
+            break;
+        }
+        n_commit[b] = n;
+        for (int32_t i = n; i < K; ++i) committed[(int64_t)b * K + i] = -1;
+        next_anchor[b] = committed[(int64_t)b * K + n - 1];
+        if (margin) margin[b] = worst;
+        free(p); free(q);
+    }
+    return rc;
 }
 
 /*
