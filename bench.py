@@ -205,6 +205,7 @@ class DeviceState:
         del host_layers
         self.logits = views[(-1, "logits")]
         self.draft = views[(-1, "draft")]
+        self.temperature = 0.0
         self.ws = B.new_workspace(B.orthrus_attend_workspace_bytes(self.layer[0]))
         Bn, K = wl.batch, wl.block
         i32 = dict(dtype=torch.int32, device=dev)
@@ -233,8 +234,27 @@ class DeviceState:
                                        self.out_a[l], self.ws)
 
     def phase_consensus(self):
-        self.B.orthrus_consensus_accept(self.logits, self.draft, self.n_commit, self.committed,
-                                        self.ar_argmax, self.next_anchor, self.cws)
+        if self.temperature > 0:
+            self.B.orthrus_consensus_sample(self.logits, self.diff_logits, self.draft, self.u_accept,
+                                            self.u_resample, self.temperature, self.n_commit,
+                                            self.committed, self.next_anchor, self.sws)
+        else:
+            self.B.orthrus_consensus_accept(self.logits, self.draft, self.n_commit, self.committed,
+                                            self.ar_argmax, self.next_anchor, self.cws)
+
+    def enable_sampling(self, temperature: float):
+        """Consensus by rejection sampling (temperature > 0): needs the diffusion view's logits
+        (drawn like the AR logits plus noise, so that drafts are accepted at a realistic rate)
+        and two uniforms per block position."""
+        B, wl = self.B, self.wl
+        g = torch.Generator().manual_seed(W.sub_seed(W.BASE_SEED, wl.name, 0, "sampling"))
+        lg = self.logits.cpu().float()
+        noise = torch.randn(lg.shape, generator=g) * (0.5 * wl.logit_std)
+        self.diff_logits = (lg + noise).to(self.logits.dtype).to(self.dev)
+        self.u_accept = torch.rand(wl.batch, wl.block, generator=g).to(self.dev)
+        self.u_resample = torch.rand(wl.batch, wl.block, generator=g).to(self.dev)
+        self.sws = B.new_workspace(B.orthrus_consensus_sample_workspace_bytes(wl.batch, wl.block, wl.vocab))
+        self.temperature = float(temperature)
 
     def phase_commit(self):
         # one launch commits the accepted rows of every layer; all layers share one length
@@ -295,6 +315,8 @@ def run_gpu(args):
     if args.no_early_launch:
         flags |= B.LAYER_NO_EARLY_LAUNCH
     st = DeviceState(wl, layers, dev, flags)
+    if args.temperature > 0:
+        st.enable_sampling(args.temperature)
     stream = torch.cuda.Stream(device=dev)
     phases = st.phases()
 
@@ -390,6 +412,7 @@ def run_gpu(args):
                    "l2": "inputs larger than L2 (distinct KV per layer)" if step_bytes > 2.5e8
                          else "L2-resident (reported, not a roofline workload)",
                    "cuda_graph": not args.no_graph, "attend_path": path,
+                   "consensus": "greedy" if args.temperature <= 0 else f"rejection sampling, T={args.temperature}",
                    "early_launch": not args.no_early_launch,
                    "early_cache_prefetch": not args.no_early_prefetch,
                    "multi_gpu": "replicas only"},
@@ -494,7 +517,8 @@ def cpu_baseline(wl, budget_s=20.0, gpu_state=None):
                                      f"the oracle (max-abs {err:.3e}, max|ref| {scale:.3e})")
                 worst = max(worst, err / scale)
                 checked += rows.shape[0]
-            if layer == 0 and not (torch.equal(gpu_state.n_commit.cpu(), cons[0]) and
+            if layer == 0 and gpu_state.temperature <= 0 and not (
+                    torch.equal(gpu_state.n_commit.cpu(), cons[0]) and
                                    torch.equal(gpu_state.committed.cpu(), cons[1])):
                 raise SystemExit("bench.py: consensus of the timed step differs from the oracle")
         layer += 1
@@ -546,6 +570,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(W.CONFIGS))
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count")
+    ap.add_argument("--temperature", type=float, default=0.0,
+                    help="> 0: the consensus phase uses rejection sampling instead of the greedy rule")
     ap.add_argument("--block", type=int, default=0,
                     help="override the block width K (the block-size sweep of Section 5)")
     ap.add_argument("--no-graph", action="store_true")

@@ -159,7 +159,32 @@ orthrus_status_t orthrus_consensus_accept(const void *ar_logits, int32_t dtype,
         void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * The same consensus for callers that cannot hand over a workspace.  (The paper has no
+ * Sampled consensus for temperature T > 0: the exact rejection sampling of Section 3.3
+ * (the speculative-sampling rule of the work cited there), which keeps the committed
+ * tokens distributed as the AR view alone would have sampled them.
+ *   p_k = softmax(ar_logits[b][k] / T),  q_k = softmax(diff_logits[b][k] / T);
+ *   draft[b][k] (drawn from q_k by the caller) is kept iff
+ *       u_accept[b][k] * q_k(draft) <= p_k(draft)      (probability min(1, p/q));
+ *   at the first k that fails, committed[b][k] is drawn from max(0, p_k - q_k),
+ *   normalised, by inverting its running sum over the vocabulary with u_resample[b][k]
+ *   (from p_k itself if that residual is empty), and verification halts;
+ *   n_commit[b] = kept drafts + 1, or K when every draft is kept;
+ *   committed[b][i] = -1 for i >= n_commit[b];  next_anchor[b] = last committed token.
+ * ar_logits, diff_logits: [B][K][V] of `dtype`; draft int32 [B][K]; u_accept, u_resample:
+ * float32 [B][K] in [0, 1), drawn by the caller (the library draws no random numbers);
+ * temperature > 0.  Softmax sums are taken in fp32 in a fixed order: results are
+ * reproducible, and differ from an exact evaluation only where a comparison is within
+ * rounding of a tie.  The commit of the accepted KV rows is orthrus_kv_append as before.
+ */
+size_t orthrus_consensus_sample_workspace_bytes(int32_t batch, int32_t block, int32_t vocab);
+orthrus_status_t orthrus_consensus_sample(const void *ar_logits, const void *diff_logits, int32_t dtype,
+        const int32_t *draft, const float *u_accept, const float *u_resample, float temperature,
+        int32_t batch, int32_t block, int32_t vocab,
+        int32_t *n_commit, int32_t *committed, int32_t *next_anchor,
+        void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The greedy consensus for callers that cannot hand over a workspace.  (The paper has no
  * counterpart to this entry point; it exists for the embedding, not for the method.)
  *
  * Who needs it: code that runs where device memory may not be allocated - a plugin that

@@ -174,8 +174,10 @@ def consensus_sample(ar_logits: torch.Tensor, diff_logits: torch.Tensor, draft: 
                      u_accept: torch.Tensor, u_resample: torch.Tensor, temperature: float):
     """Sampled consensus for T > 0 (the rejection-sampling rule of Section 3.3).
     u_accept, u_resample: [B][K] in [0, 1).  Returns (n_commit [B], committed [B][K],
-    next_anchor [B]) int32 and margin [B] float64 (distance of the nearest decision
-    from flipping, relative)."""
+    next_anchor [B]) int32 and margin [B][2] float64: [:, 0] the relative distance of the
+    nearest accept test from flipping, [:, 1] the distance of the resampling point from
+    the edges of the chosen token's residual mass, as a fraction of that mass (inf if no
+    token was resampled)."""
     _check(ar_logits, "ar_logits")
     _check(diff_logits, "diff_logits")
     _check(draft, "draft")
@@ -189,7 +191,7 @@ def consensus_sample(ar_logits: torch.Tensor, diff_logits: torch.Tensor, draft: 
     n = torch.empty(B, dtype=torch.int32)
     com = torch.empty((B, K), dtype=torch.int32)
     nxt = torch.empty(B, dtype=torch.int32)
-    margin = torch.empty(B, dtype=torch.float64)
+    margin = torch.empty((B, 2), dtype=torch.float64)
     rc = lib().oracle_consensus_sample(ar_logits.data_ptr(), diff_logits.data_ptr(),
                                        _DTYPE_CODE[ar_logits.dtype], draft.data_ptr(),
                                        ua.data_ptr(), ur.data_ptr(), float(temperature), B, K, V,

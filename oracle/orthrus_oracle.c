@@ -255,10 +255,11 @@ int oracle_consensus_accept(const void *logits, int dtype, const int32_t *draft,
  *
  * u_accept, u_resample: [B][K] doubles in [0, 1), supplied by the caller.
  * Outputs: n_commit [B], committed [B][K] (-1 beyond n), next_anchor [B], and
- * margin [B] (optional): how far the nearest decision of sequence b was from
- * flipping, relative to the quantities compared (min over the accept tests taken
- * of |u*q(y) - p(y)| / max(p(y), u*q(y)) and, if a token was resampled, of the
- * distance of u*total to the two running sums that bracket it, over total).
+ * margin [B][2] (optional): how far the decisions of sequence b were from flipping.
+ * margin[b][0] = min over the accept tests taken of |u*q(y) - p(y)| / max(p(y), u*q(y));
+ * margin[b][1] = if a token was resampled, the distance of u*total to the nearer of the
+ * two running sums that bracket it, as a fraction of the chosen token's own residual
+ * mass (0.5 = dead centre), else infinity.
  */
 int oracle_consensus_sample(const void *ar_logits, const void *diff_logits, int dtype,
                             const int32_t *draft, const double *u_accept,
@@ -279,7 +280,7 @@ int oracle_consensus_sample(const void *ar_logits, const void *diff_logits, int 
             rc = -1;
             continue;
         }
-        double worst = INFINITY;
+        double worst = INFINITY, worst_pick = INFINITY;
         int32_t n = 0;
         for (int32_t k = 0; k < K; ++k) {
             const int64_t row = ((int64_t)b * K + k) * V;
@@ -332,9 +333,9 @@ int oracle_consensus_sample(const void *ar_logits, const void *diff_logits, int 
                 prev = run;
             }
             {
-                const double lo = fabs(target - prev) / total, hi = fabs(run - target) / total;
-                const double m2 = lo < hi ? lo : hi;
-                if (m2 < worst) worst = m2;
+                const double width = run - prev;
+                const double lo = fabs(target - prev), hi = fabs(run - target);
+                worst_pick = width > 0.0 ? (lo < hi ? lo : hi) / width : 0.0;
             }
             committed[(int64_t)b * K + n] = z;
             ++n;
@@ -343,7 +344,7 @@ int oracle_consensus_sample(const void *ar_logits, const void *diff_logits, int 
         n_commit[b] = n;
         for (int32_t i = n; i < K; ++i) committed[(int64_t)b * K + i] = -1;
         next_anchor[b] = committed[(int64_t)b * K + n - 1];
-        if (margin) margin[b] = worst;
+        if (margin) { margin[2 * b] = worst; margin[2 * b + 1] = worst_pick; }
         free(p); free(q);
     }
     return rc;

@@ -24,7 +24,8 @@ EXPORTS = [
     "orthrus_attend_workspace_bytes", "orthrus_workspace_init",
     "orthrus_diffusion_block_attend", "orthrus_ar_verify_attend",
     "orthrus_consensus_workspace_bytes", "orthrus_consensus_accept",
-    "orthrus_consensus_accept_static",
+    "orthrus_consensus_accept_static", "orthrus_consensus_sample_workspace_bytes",
+    "orthrus_consensus_sample",
     "orthrus_kv_append", "orthrus_kv_append_layers", "orthrus_read_status", "orthrus_set_path", "orthrus_last_path",
     "orthrus_launch_count", "orthrus_status_string", "orthrus_version",
 ]
@@ -73,6 +74,11 @@ def _load() -> ctypes.CDLL:
     lib.orthrus_consensus_accept.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.orthrus_consensus_accept_static.restype = ctypes.c_int
     lib.orthrus_consensus_accept_static.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.orthrus_consensus_sample_workspace_bytes.restype = sz
+    lib.orthrus_consensus_sample_workspace_bytes.argtypes = [i32, i32, i32]
+    lib.orthrus_consensus_sample.restype = ctypes.c_int
+    lib.orthrus_consensus_sample.argtypes = [vp, vp, i32, vp, vp, vp, ctypes.c_float, i32, i32, i32,
+                                             vp, vp, vp, vp, sz, vp]
     lib.orthrus_kv_append.restype = ctypes.c_int
     lib.orthrus_kv_append.argtypes = [LP, vp, vp, vp, i32, vp, sz, vp]
     lib.orthrus_kv_append_layers.restype = ctypes.c_int
@@ -170,6 +176,24 @@ def orthrus_consensus_accept(ar_logits, draft, n_commit, committed, ar_argmax, n
         _ptr(ar_logits), dtype_code(ar_logits.dtype), _ptr(draft), B, K, V, _ptr(n_commit),
         _ptr(committed), _ptr(ar_argmax), _ptr(next_anchor), _ptr(workspace), workspace.numel(),
         _stream(stream)), "orthrus_consensus_accept")
+
+
+def orthrus_consensus_sample_workspace_bytes(batch: int, block: int, vocab: int) -> int:
+    return int(_lib.orthrus_consensus_sample_workspace_bytes(batch, block, vocab))
+
+
+def orthrus_consensus_sample(ar_logits, diff_logits, draft, u_accept, u_resample, temperature: float,
+                             n_commit, committed, next_anchor, workspace, stream=None) -> None:
+    """Sampled consensus for T > 0; u_accept / u_resample are float32 [B][K] device tensors."""
+    B, K, V = ar_logits.shape
+    if diff_logits.shape != ar_logits.shape or diff_logits.dtype != ar_logits.dtype:
+        raise TypeError("the two logit tensors must agree in shape and dtype")
+    if u_accept.dtype != torch.float32 or u_resample.dtype != torch.float32:
+        raise TypeError("the uniforms must be float32")
+    _check(_lib.orthrus_consensus_sample(
+        _ptr(ar_logits), _ptr(diff_logits), dtype_code(ar_logits.dtype), _ptr(draft), _ptr(u_accept),
+        _ptr(u_resample), float(temperature), B, K, V, _ptr(n_commit), _ptr(committed), _ptr(next_anchor),
+        _ptr(workspace), workspace.numel(), _stream(stream)), "orthrus_consensus_sample")
 
 
 STATIC_CONSENSUS_SCRATCH_BYTES = 65536

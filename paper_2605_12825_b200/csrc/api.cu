@@ -276,6 +276,40 @@ orthrus_status_t orthrus_consensus_accept(const void *ar_logits, int32_t dtype, 
     return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
 }
 
+size_t orthrus_consensus_sample_workspace_bytes(int32_t batch, int32_t block, int32_t vocab)
+{
+    if (batch < 1 || block < 1 || vocab < 1) return 0;
+    return kHeaderBytes + sample_workspace_bytes(batch, block, vocab);
+}
+
+orthrus_status_t orthrus_consensus_sample(const void *ar_logits, const void *diff_logits, int32_t dtype,
+        const int32_t *draft, const float *u_accept, const float *u_resample, float temperature,
+        int32_t batch, int32_t block, int32_t vocab, int32_t *n_commit, int32_t *committed,
+        int32_t *next_anchor, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (batch < 1 || block < 1 || vocab < 1 || !(temperature > 0.f) || std::isinf(temperature))
+        return ORTHRUS_ERR_INVALID_ARG;
+    if (dtype != ORTHRUS_BF16 && dtype != ORTHRUS_FP32) return ORTHRUS_ERR_UNSUPPORTED;
+    if (block > 1024 || (long long)batch * block > 65535) return ORTHRUS_ERR_UNSUPPORTED;
+    if (!ar_logits || !diff_logits || !draft || !u_accept || !u_resample || !n_commit || !committed ||
+        !next_anchor || !workspace)
+        return ORTHRUS_ERR_INVALID_ARG;
+    const size_t es = dtype == ORTHRUS_FP32 ? 4 : 2;
+    if (((reinterpret_cast<uintptr_t>(ar_logits) | reinterpret_cast<uintptr_t>(diff_logits)) & (es - 1)) ||
+        !aligned16(workspace) ||
+        ((reinterpret_cast<uintptr_t>(draft) | reinterpret_cast<uintptr_t>(u_accept) |
+          reinterpret_cast<uintptr_t>(u_resample) | reinterpret_cast<uintptr_t>(n_commit) |
+          reinterpret_cast<uintptr_t>(committed) | reinterpret_cast<uintptr_t>(next_anchor)) & 3))
+        return ORTHRUS_ERR_INVALID_ARG;
+    if (workspace_bytes < orthrus_consensus_sample_workspace_bytes(batch, block, vocab))
+        return ORTHRUS_ERR_WORKSPACE;
+    cudaError_t e = launch_consensus_sample(ar_logits, diff_logits, dtype, draft, u_accept, u_resample,
+                                            temperature, batch, block, vocab, n_commit, committed, next_anchor,
+                                            static_cast<unsigned char *>(workspace) + kHeaderBytes,
+                                            static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+}
+
 orthrus_status_t orthrus_consensus_accept_static(const void *ar_logits, int32_t dtype,
         const int32_t *draft, int32_t batch, int32_t block, int32_t vocab, int32_t *n_commit,
         int32_t *committed, int32_t *ar_argmax, int32_t *next_anchor, void *stream)

@@ -75,6 +75,12 @@ cudaError_t launch_kv_append(const orthrus_layer_t &L, const void *k_blk, const 
                              const int32_t *n_commit, int update_len, int32_t *status,
                              cudaStream_t st);
 
+size_t sample_workspace_bytes(int B, int K, int V);
+cudaError_t launch_consensus_sample(const void *ar_logits, const void *diff_logits, int dtype, const int32_t *draft,
+                                    const float *u_accept, const float *u_resample, float temperature, int B, int K,
+                                    int V, int32_t *n_commit, int32_t *committed, int32_t *next_anchor, void *ws,
+                                    cudaStream_t st);
+
 struct AppendLayer { void *k_cache, *v_cache; const void *k_blk, *v_blk; int32_t *cache_len; };
 cudaError_t launch_kv_append_layers(const orthrus_layer_t &shape, const AppendLayer *layers, int n_layers,
                                     int32_t *const *len_arrays, int n_len_arrays,
