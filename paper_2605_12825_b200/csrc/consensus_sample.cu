@@ -129,17 +129,20 @@ __global__ void __launch_bounds__(kThreads) sample_stats_kernel(const T *la, con
     if (vec) {                                  // seg_len and V are multiples of N, rows are 16-byte aligned
         const uint4 *va = reinterpret_cast<const uint4 *>(ra + start), *vd = reinterpret_cast<const uint4 *>(rd + start);
         const int n_vec = (end - start) / N;
-        for (int v = threadIdx.x; v < n_vec; v += 2 * kThreads) {
-            const bool two = v + kThreads < n_vec;
-            const uint4 a0 = __ldg(va + v), d0 = __ldg(vd + v);
-            uint4 a1 = a0, d1 = d0;
-            if (two) { a1 = __ldg(va + v + kThreads); d1 = __ldg(vd + v + kThreads); }
-            float x[N];
-            Elem<T>::unpack(a0, x); absorb_vec<N>(a, x, c);
-            Elem<T>::unpack(d0, x); absorb_vec<N>(d, x, c);
-            if (two) {
-                Elem<T>::unpack(a1, x); absorb_vec<N>(a, x, c);
-                Elem<T>::unpack(d1, x); absorb_vec<N>(d, x, c);
+        for (int v = threadIdx.x; v < n_vec; v += 4 * kThreads) {     // up to 8 loads in flight per thread
+            uint4 av[4], dv[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int w = min(v + k * kThreads, n_vec - 1);
+                av[k] = __ldg(va + w); dv[k] = __ldg(vd + w);
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (v + k * kThreads < n_vec) {
+                    float x[N];
+                    Elem<T>::unpack(av[k], x); absorb_vec<N>(a, x, c);
+                    Elem<T>::unpack(dv[k], x); absorb_vec<N>(d, x, c);
+                }
             }
         }
     } else {
@@ -153,7 +156,7 @@ __global__ void __launch_bounds__(kThreads) sample_stats_kernel(const T *la, con
     if (threadIdx.x == 0) parts[(long long)row * gridDim.x + seg] = StatPart{a.m, d.m, a.s, d.s};
 }
 
-struct RowStat { float ma, md; double za, zd; int row; int pad; };   // of the first rejected row; row = -1: none
+struct RowStat { float ma, md; double inv_za, inv_zd; int row; int pad; };   // of the first rejected row (1 / sums); row = -1: none
 
 // 2. per sequence: fold the segments, take the accept tests, find the first failure
 template <typename T>
@@ -192,7 +195,7 @@ __global__ void sample_decide_kernel(const T *la, const T *ld, const StatPart *p
         RowStat st;
         st.row = j < K ? j : -1;
         const StatPart f = folded[j < K ? j : 0];
-        st.ma = f.ma; st.za = f.sa; st.md = f.md; st.zd = f.sd;
+        st.ma = f.ma; st.inv_za = 1.0 / f.sa; st.md = f.md; st.inv_zd = 1.0 / f.sd;
         st.pad = 0;
         stat[b] = st;
         if (j >= K) next_anchor[b] = draft[(long long)b * K + K - 1];
@@ -200,8 +203,8 @@ __global__ void sample_decide_kernel(const T *la, const T *ld, const StatPart *p
 }
 
 __device__ inline void residual_of(float xa, float xd, float c, const RowStat &st, double &r, double &p) {
-    p = (double)ex2f(xa * c - st.ma) / st.za;
-    const double q = (double)ex2f(xd * c - st.md) / st.zd;
+    p = (double)ex2f(xa * c - st.ma) * st.inv_za;
+    const double q = (double)ex2f(xd * c - st.md) * st.inv_zd;
     r = fmax(p - q, 0.0);
 }
 
@@ -322,7 +325,7 @@ __global__ void __launch_bounds__(kThreads) sample_pick_kernel(const T *la, cons
 int sample_stat_segments(int B, int K, int V)
 {
     const long long rows = (long long)B * K;
-    long long want = (4LL * kNumSMs + rows - 1) / rows;
+    long long want = (8LL * kNumSMs + rows - 1) / rows;           // more CTAs than fit at once, for balance
     const long long max_by_len = (V + 4095) / 4096;
     if (want > max_by_len) want = max_by_len;
     return (int)(want < 1 ? 1 : want);
