@@ -114,3 +114,46 @@ def test_generation_bf16_tcgen05_shapes():
     assert ties <= 2
     assert 1.5 < mean_n < 4.5
     assert binding().orthrus_last_path() == "tcgen05"
+
+
+def test_sampled_generation_loop_fp32():
+    """Temperature 1: drafts are SAMPLED from the diffusion view's own logits, verified by
+    the AR view and reconciled by rejection sampling.  Every cycle's outcome equals the
+    oracle's on the GPU's own logits (up to near ties), and the cache grows by n."""
+    b = binding()
+    b.orthrus_set_path("auto")
+    layers, hidden, n_q, n_kv, d, ffn, vocab = 2, 128, 4, 2, 32, 256, 400
+    B, T_prompt, K, cycles, temp = 3, 30, 6, 10, 1.0
+    cap = T_prompt + cycles * K + 8
+    g = torch.Generator().manual_seed(23)
+    prompt = torch.randint(0, vocab, (B, T_prompt), generator=g).cuda()
+    dec = Decoder(b, layers, hidden, n_q, n_kv, d, ffn, vocab, torch.float32, B, cap, K, seed=4)
+    anchor = dec.prefill(prompt)
+    sws = b.new_workspace(b.orthrus_consensus_sample_workspace_bytes(B, K, vocab))
+    i32 = dict(dtype=torch.int32, device="cuda")
+    n_c, com, nxt = torch.zeros(B, **i32), torch.zeros(B, K, **i32), torch.zeros(B, **i32)
+    total, undecided = 0, 0
+    for _ in range(cycles):
+        blk = torch.full((B, K), vocab, dtype=torch.int32, device="cuda")
+        blk[:, 0] = anchor
+        d_logits, _, _ = dec.forward_block(blk, "diff", K)
+        # row i of the diffusion pass proposes the token after block position i
+        q = torch.softmax(d_logits.float().cpu() / temp, -1)
+        draft = torch.multinomial(q.view(-1, vocab), 1, generator=g).view(B, K).to(torch.int32)
+        ar_in = torch.cat([anchor.view(B, 1), draft[:, :K - 1].cuda()], dim=1)
+        logits, ks, vs = dec.forward_block(ar_in, "ar", K)
+        ua, ur = torch.rand(B, K, generator=g), torch.rand(B, K, generator=g)
+        len_before = dec.cache_len.cpu().clone()
+        b.orthrus_consensus_sample(logits, d_logits, draft.cuda(), ua.cuda(), ur.cuda(), temp, n_c, com, nxt, sws)
+        rn, rcom, rnxt, margin = oracle.consensus_sample(logits.cpu(), d_logits.cpu(), draft, ua.double(),
+                                                         ur.double(), temp)
+        ok = (margin[:, 0] > 1e-4) & (margin[:, 1] > 1e-2)
+        undecided += int((~ok).sum())
+        assert torch.equal(n_c.cpu()[ok], rn[ok]) and torch.equal(com.cpu()[ok], rcom[ok])
+        assert torch.equal(nxt.cpu()[ok], rnxt[ok])
+        assert int(n_c.min()) >= 1 and int(n_c.max()) <= K
+        dec.commit(ks, vs, n_c, K)
+        assert torch.equal(dec.cache_len.cpu(), len_before + n_c.cpu())
+        anchor = nxt.clone()
+        total += int(n_c.sum())
+    assert undecided <= 2 and total >= cycles * B
