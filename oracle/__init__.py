@@ -74,6 +74,12 @@ def lib() -> ctypes.CDLL:
                                                  ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                                                  ctypes.c_void_p, ctypes.c_void_p]
         _lib.oracle_kv_append.restype = ctypes.c_int
+        _lib.oracle_lm_head_argmax.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                                               ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
+                                               ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
+        _lib.oracle_accept_rule.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
+                                            ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                            ctypes.c_void_p]
         _lib.oracle_kv_append.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                           ctypes.c_int32, ctypes.c_int64, ctypes.c_int,
                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -199,6 +205,60 @@ def consensus_sample(ar_logits: torch.Tensor, diff_logits: torch.Tensor, draft: 
     if rc != 0:
         raise RuntimeError(f"oracle_consensus_sample failed ({rc})")
     return n, com, nxt, margin
+
+
+def lm_head_argmax(hidden: torch.Tensor, lm_head: torch.Tensor, rows: Optional[torch.Tensor] = None
+                   ) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Greedy token of rows of hidden [R][H] under the LM head [V][H] (logit = dot product in
+    fp64).  rows: optional int32 list of row numbers (default: all).  Returns (arg [n] int32,
+    top2 [n][2] float64 = the largest logit and the largest among the other ids)."""
+    _check(hidden, "hidden")
+    _check(lm_head, "lm_head")
+    R, H = hidden.shape
+    V, H2 = lm_head.shape
+    if H2 != H or hidden.dtype != lm_head.dtype:
+        raise ValueError("hidden [R][H] and lm_head [V][H] must agree in H and dtype")
+    if rows is not None:
+        rows = _check(rows.to(torch.int32).contiguous(), "rows")
+        if rows.numel() and (int(rows.min()) < 0 or int(rows.max()) >= R):
+            raise ValueError("row out of range")
+    n = R if rows is None else rows.numel()
+    arg = torch.empty(n, dtype=torch.int32)
+    top2 = torch.empty((n, 2), dtype=torch.float64)
+    rc = lib().oracle_lm_head_argmax(hidden.data_ptr(), lm_head.data_ptr(), _DTYPE_CODE[hidden.dtype],
+                                     None if rows is None else rows.data_ptr(), n, V, H,
+                                     arg.data_ptr(), top2.data_ptr())
+    if rc != 0:
+        raise RuntimeError(f"oracle_lm_head_argmax failed ({rc})")
+    return arg, top2
+
+
+def accept_rule(g: torch.Tensor, draft: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    """The halt/commit rule of Section 3.3 on given greedy tokens g [B][K] int32.
+    Returns (n_commit [B], committed [B][K], next_anchor [B])."""
+    _check(g, "g")
+    _check(draft, "draft")
+    B, K = g.shape
+    if g.dtype != torch.int32 or draft.dtype != torch.int32 or tuple(draft.shape) != (B, K):
+        raise ValueError("g and draft must be int32 [B][K]")
+    n = torch.empty(B, dtype=torch.int32)
+    com = torch.empty((B, K), dtype=torch.int32)
+    nxt = torch.empty(B, dtype=torch.int32)
+    rc = lib().oracle_accept_rule(g.data_ptr(), draft.data_ptr(), B, K, n.data_ptr(), com.data_ptr(),
+                                  nxt.data_ptr())
+    if rc != 0:
+        raise RuntimeError(f"oracle_accept_rule failed ({rc})")
+    return n, com, nxt
+
+
+def lm_head_consensus(hidden: torch.Tensor, lm_head: torch.Tensor, draft: torch.Tensor):
+    """Greedy consensus from the AR view's last hidden states [B][K][H] and the LM head [V][H].
+    Returns (n_commit, committed, ar_argmax [B][K], next_anchor) int32 and top2 [B][K][2]."""
+    B, K, H = hidden.shape
+    arg, top2 = lm_head_argmax(hidden.reshape(B * K, H), lm_head)
+    g = arg.reshape(B, K).contiguous()
+    n, com, nxt = accept_rule(g, draft)
+    return n, com, g, nxt, top2.reshape(B, K, 2)
 
 
 def kv_append(k_cache, v_cache, cache_len, k_blk, v_blk, n_commit, update_len: bool = True) -> int:

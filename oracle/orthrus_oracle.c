@@ -23,7 +23,9 @@
  * model, byte-level append checks; for the sampled consensus: the committed token
  * follows the AR distribution, acceptance rate 1 - total variation, reduction to
  * the greedy rule at low temperature, library inverse-CDF on the degenerate
- * cases).  Nothing is "parity unpinned".
+ * cases) and tests/test_oracle_lm_head_pins.py (planted maxima, exact-integer
+ * logits against the logits-based rule, the library matrix product, ties, a
+ * transposition trap).  Nothing is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -224,6 +226,74 @@ int oracle_consensus_accept(const void *logits, int dtype, const int32_t *draft,
     }
     for (int32_t b = 0; b < B; ++b) {
         const int32_t *g = ar_argmax + (int64_t)b * K;
+        const int32_t *y = draft + (int64_t)b * K;
+        int32_t m = 0;
+        while (m < K && y[m] == g[m]) ++m;
+        const int32_t n = (m + 1 < K) ? m + 1 : K;
+        n_commit[b] = n;
+        for (int32_t i = 0; i < K; ++i)
+            committed[(int64_t)b * K + i] = (i < n) ? g[i] : -1;
+        next_anchor[b] = g[n - 1];
+    }
+    return 0;
+}
+
+/*
+ * Greedy tokens straight from the last hidden states (the step that produces the
+ * logits Eq. 8 takes the argmax of: logits[r][v] = sum_c hidden[r][c] * lm_head[v][c],
+ * the shared LM head of Section 3.1 applied to row r of the AR view's final hidden
+ * states).  Every product and sum is carried in double; nothing is rounded to a
+ * storage type before the comparison.
+ *
+ * rows == NULL: all n_rows rows 0..n_rows-1; otherwise rows[j] names the row of
+ * `hidden` that output j is computed from (for sampled checks at full size).
+ * Outputs per listed row: arg (smallest id attaining the maximum; a NaN never
+ * wins) and top2 = (largest logit, largest logit among the other ids; -inf when
+ * V == 1), from which a caller judges how close the decision was.
+ */
+int oracle_lm_head_argmax(const void *hidden, const void *lm_head, int dtype,
+                          const int32_t *rows, int32_t n_rows, int32_t V, int32_t H,
+                          int32_t *arg, double *top2)
+{
+    if (n_rows < 0 || V <= 0 || H <= 0) return -2;
+    int rc = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t j = 0; j < n_rows; ++j) {
+        const int64_t r = rows ? rows[j] : j;
+        double *x = (double *)malloc((size_t)H * sizeof(double));
+        if (!x) {
+#pragma omp critical
+            rc = -4;
+            continue;
+        }
+        for (int32_t c = 0; c < H; ++c) x[c] = load_elem(hidden, dtype, r * H + c);
+        double best = -INFINITY, second = -INFINITY;
+        int32_t a = 0;
+        for (int32_t v = 0; v < V; ++v) {
+            double s = 0.0;
+            for (int32_t c = 0; c < H; ++c) s += x[c] * load_elem(lm_head, dtype, (int64_t)v * H + c);
+            if (s > best) { second = best; best = s; a = v; }
+            else if (s > second) second = s;
+        }
+        arg[j] = a;
+        top2[2 * j] = best;
+        top2[2 * j + 1] = second;
+        free(x);
+    }
+    return rc;
+}
+
+/*
+ * The accept rule of oracle_consensus_accept applied to given greedy tokens g [B][K]
+ * (Eq. 8 and the halt/commit rule of Section 3.3): n = min(m + 1, K) with m the number
+ * of leading drafts equal to g, committed = g_0..g_{n-1} (-1 beyond), next anchor g_{n-1}.
+ */
+int oracle_accept_rule(const int32_t *g_all, const int32_t *draft, int32_t B, int32_t K,
+                       int32_t *n_commit, int32_t *committed, int32_t *next_anchor)
+{
+    if (B < 0 || K <= 0) return -2;
+    for (int32_t b = 0; b < B; ++b) {
+        const int32_t *g = g_all + (int64_t)b * K;
         const int32_t *y = draft + (int64_t)b * K;
         int32_t m = 0;
         while (m < K && y[m] == g[m]) ++m;

@@ -1,6 +1,6 @@
 """The oracle's C code under AddressSanitizer and UndefinedBehaviorSanitizer: a small
 run of every entry point (ragged batch, empty prefix, both views, weights requested,
-consensus with ties and specials, append with an overflowing sequence) in a child
+consensus with ties and specials, the LM-head argmax, append with an overflowing sequence) in a child
 process, which must finish without a sanitizer report."""
 import os
 import subprocess
@@ -38,6 +38,11 @@ rc = oracle.kv_append(kc, vc, lens, kb, vb, torch.tensor([1, 5, 5], dtype=torch.
 assert rc == 0 and lens.tolist() == [1, 22, 40]
 rc = oracle.kv_append(kc, vc, lens, kb, vb, torch.tensor([1, 1, 1], dtype=torch.int32))
 assert rc != 0 and lens.tolist() == [2, 23, 40]
+hid, W = mk(B, K, 24), mk(77, 24)
+n2, com2, g2, nxt2, top2 = oracle.lm_head_consensus(hid, W, draft % 77)
+assert 1 <= int(n2.min()) and int(n2.max()) <= K and bool((top2[..., 0] >= top2[..., 1]).all())
+a3, _ = oracle.lm_head_argmax(hid.reshape(B * K, 24), W, torch.tensor([14, 0], dtype=torch.int32))
+assert a3.tolist() == [int(g2[2, 4]), int(g2[0, 0])]
 print("sanitized run ok")
 '''
 
