@@ -216,6 +216,32 @@ orthrus_status_t orthrus_consensus_accept_static(const void *ar_logits, int32_t 
         void *stream);
 
 /*
+ * Greedy consensus straight from the AR view's last hidden states (the step before Eq. 8
+ * fused into it): with the shared LM head of Section 3.1,
+ *   logits[b][i][v] = sum_c hidden[b][i][c] * lm_head[v][c],
+ * the greedy tokens g[b][i] = argmax_v logits[b][i][v] (smallest id on ties, a NaN never
+ * wins) and then the accept rule of orthrus_consensus_accept on g.  The logits are never
+ * written to memory.  Products of the bf16 operands are accumulated in fp32 on the tensor
+ * cores and compared as fp32 sums (they are not rounded to bf16 first, so a near-tie can
+ * resolve differently from the two-step path that stores bf16 logits).
+ *
+ * hidden   device [batch][block][hidden_dim] bf16 (final-norm output of the AR view)
+ * lm_head  device [vocab][hidden_dim] bf16, one row per vocabulary entry
+ * Both 16-byte aligned; hidden_dim a multiple of 8.  draft and the four outputs as for
+ * orthrus_consensus_accept.  Only ORTHRUS_BF16 is supported (anything else, or a driver
+ * without tensor-map support: ORTHRUS_ERR_UNSUPPORTED).  `workspace`: at least
+ * orthrus_lm_head_consensus_workspace_bytes(batch, block, vocab) bytes, 16-byte aligned,
+ * header initialised by orthrus_workspace_init; a wait inside the kernel that does not end
+ * reports ORTHRUS_DEV_WAIT_TIMEOUT through orthrus_read_status and leaves the outputs of
+ * that call undefined.  Two launches; nothing is allocated and the stream is not synchronised.
+ */
+size_t orthrus_lm_head_consensus_workspace_bytes(int32_t batch, int32_t block, int32_t vocab);
+orthrus_status_t orthrus_lm_head_consensus(const void *hidden, const void *lm_head, int32_t dtype,
+        int32_t hidden_dim, const int32_t *draft, int32_t batch, int32_t block, int32_t vocab,
+        int32_t *n_commit, int32_t *committed, int32_t *ar_argmax, int32_t *next_anchor,
+        void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * KV commit (Figure 2(b); last paragraph of Section 3.3): for every sequence b,
  * KV head h and i < n_commit[b],
  *   k_cache[b][h][P_b + i] = k_ar_blk[b][i][h]   (likewise v),

@@ -26,6 +26,7 @@ EXPORTS = [
     "orthrus_consensus_workspace_bytes", "orthrus_consensus_accept",
     "orthrus_consensus_accept_static", "orthrus_consensus_sample_workspace_bytes",
     "orthrus_consensus_sample",
+    "orthrus_lm_head_consensus_workspace_bytes", "orthrus_lm_head_consensus",
     "orthrus_kv_append", "orthrus_kv_append_layers", "orthrus_read_status", "orthrus_set_path", "orthrus_last_path",
     "orthrus_launch_count", "orthrus_status_string", "orthrus_version",
 ]
@@ -79,6 +80,10 @@ def _load() -> ctypes.CDLL:
     lib.orthrus_consensus_sample.restype = ctypes.c_int
     lib.orthrus_consensus_sample.argtypes = [vp, vp, i32, vp, vp, vp, ctypes.c_float, i32, i32, i32,
                                              vp, vp, vp, vp, sz, vp]
+    lib.orthrus_lm_head_consensus_workspace_bytes.restype = sz
+    lib.orthrus_lm_head_consensus_workspace_bytes.argtypes = [i32, i32, i32]
+    lib.orthrus_lm_head_consensus.restype = ctypes.c_int
+    lib.orthrus_lm_head_consensus.argtypes = [vp, vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.orthrus_kv_append.restype = ctypes.c_int
     lib.orthrus_kv_append.argtypes = [LP, vp, vp, vp, i32, vp, sz, vp]
     lib.orthrus_kv_append_layers.restype = ctypes.c_int
@@ -210,6 +215,22 @@ def orthrus_consensus_accept_static(ar_logits, draft, n_commit, committed, ar_ar
         _ptr(ar_logits), dtype_code(ar_logits.dtype), _ptr(draft), B, K, V, _ptr(n_commit),
         _ptr(committed), _ptr(ar_argmax), _ptr(next_anchor), _stream(stream)),
         "orthrus_consensus_accept_static")
+
+
+def orthrus_lm_head_consensus_workspace_bytes(batch: int, block: int, vocab: int) -> int:
+    return int(_lib.orthrus_lm_head_consensus_workspace_bytes(batch, block, vocab))
+
+
+def orthrus_lm_head_consensus(hidden, lm_head, draft, n_commit, committed, ar_argmax, next_anchor,
+                              workspace, stream=None) -> None:
+    """Greedy consensus from the last hidden states [B][K][H] and the LM head [V][H] (bf16);
+    the logits are never materialised."""
+    B, K, H = hidden.shape
+    V = lm_head.shape[0]
+    _check(_lib.orthrus_lm_head_consensus(
+        _ptr(hidden), _ptr(lm_head), dtype_code(hidden.dtype), H, _ptr(draft), B, K, V, _ptr(n_commit),
+        _ptr(committed), _ptr(ar_argmax), _ptr(next_anchor), _ptr(workspace), workspace.numel(),
+        _stream(stream)), "orthrus_lm_head_consensus")
 
 
 def orthrus_kv_append(layer: Layer, k_ar_blk, v_ar_blk, n_commit, update_len: bool = True,

@@ -334,6 +334,42 @@ orthrus_status_t orthrus_consensus_accept_static(const void *ar_logits, int32_t 
     return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
 }
 
+size_t orthrus_lm_head_consensus_workspace_bytes(int32_t batch, int32_t block, int32_t vocab)
+{
+    if (batch < 1 || block < 1 || vocab < 1) return 0;
+    return kHeaderBytes + (size_t)batch * block * lm_head_vocab_tiles(vocab) * sizeof(ArgPart);
+}
+
+orthrus_status_t orthrus_lm_head_consensus(const void *hidden, const void *lm_head, int32_t dtype,
+        int32_t hidden_dim, const int32_t *draft, int32_t batch, int32_t block, int32_t vocab,
+        int32_t *n_commit, int32_t *committed, int32_t *ar_argmax, int32_t *next_anchor,
+        void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (batch < 1 || block < 1 || vocab < 1 || hidden_dim < 1) return ORTHRUS_ERR_INVALID_ARG;
+    if (dtype != ORTHRUS_BF16) return ORTHRUS_ERR_UNSUPPORTED;
+    if (block > 1024 || (long long)batch * block > 65535 || vocab > (1 << 24) || (hidden_dim & 7))
+        return ORTHRUS_ERR_UNSUPPORTED;
+    if (!hidden || !lm_head || !draft || !n_commit || !committed || !ar_argmax || !next_anchor || !workspace)
+        return ORTHRUS_ERR_INVALID_ARG;
+    if (!aligned16(hidden) || !aligned16(lm_head) || !aligned16(workspace) ||
+        ((reinterpret_cast<uintptr_t>(draft) | reinterpret_cast<uintptr_t>(n_commit) |
+          reinterpret_cast<uintptr_t>(committed) | reinterpret_cast<uintptr_t>(ar_argmax) |
+          reinterpret_cast<uintptr_t>(next_anchor)) & 3))
+        return ORTHRUS_ERR_INVALID_ARG;
+    if (workspace_bytes < orthrus_lm_head_consensus_workspace_bytes(batch, block, vocab))
+        return ORTHRUS_ERR_WORKSPACE;
+    if (!lm_head_supported()) return ORTHRUS_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ArgPart *parts = reinterpret_cast<ArgPart *>(static_cast<unsigned char *>(workspace) + kHeaderBytes);
+    cudaError_t e = launch_lm_head_argmax(hidden, lm_head, batch * block, vocab, hidden_dim, parts,
+                                          static_cast<int32_t *>(workspace), st);
+    if (e == cudaErrorNotSupported) return ORTHRUS_ERR_UNSUPPORTED;
+    if (e == cudaSuccess)
+        e = launch_consensus_finalize_wide(parts, lm_head_vocab_tiles(vocab), draft, batch, block, n_commit,
+                                           committed, ar_argmax, next_anchor, st);
+    return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+}
+
 orthrus_status_t orthrus_kv_append(const orthrus_layer_t *layer, const void *k_ar_blk,
         const void *v_ar_blk, const int32_t *n_commit, int32_t update_len, void *workspace,
         size_t workspace_bytes, void *stream)

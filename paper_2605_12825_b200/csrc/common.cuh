@@ -66,6 +66,14 @@ cudaError_t launch_consensus(const void *logits, int dtype, const int32_t *draft
                              int V, int32_t *n_commit, int32_t *committed, int32_t *ar_argmax,
                              int32_t *next_anchor, void *partials, int n_seg, cudaStream_t st);
 int consensus_segments(int B, int K, int V);
+struct ArgPart { float v; int idx; };    // the best (value, id) of one stretch of a row
+cudaError_t launch_consensus_finalize_wide(const ArgPart *parts, int n_seg, const int32_t *draft, int B,
+                                           int K, int32_t *n_commit, int32_t *committed,
+                                           int32_t *ar_argmax, int32_t *next_anchor, cudaStream_t st);
+int lm_head_vocab_tiles(int V);
+bool lm_head_supported();
+cudaError_t launch_lm_head_argmax(const void *hidden, const void *lm_head, int R, int V, int H,
+                                  ArgPart *parts, int32_t *status, cudaStream_t st);
 size_t static_consensus_scratch_needed(int B, int K, int V);
 cudaError_t launch_consensus_static(const void *logits, int dtype, const int32_t *draft, int B, int K,
                                     int V, int32_t *n_commit, int32_t *committed, int32_t *ar_argmax,

@@ -7,8 +7,6 @@
 namespace orthrus {
 namespace {
 
-struct ArgPart { float v; int idx; };
-
 __device__ inline bool better(float v, int i, float bv, int bi) {
     return v > bv || (v == bv && i < bi);
 }
@@ -153,7 +151,58 @@ __global__ void consensus_finalize_kernel(const ArgPart *parts, int n_seg, const
         committed[(long long)b * K + i] = i < n ? g[i] : -1;
 }
 
+// The same with many partials per row (one per vocabulary tile of the fused LM head): a warp
+// per row folds them, lanes striding over the tiles.
+__global__ void __launch_bounds__(256) consensus_finalize_wide_kernel(
+        const ArgPart *parts, int n_seg, const int32_t *draft, int K, int32_t *n_commit,
+        int32_t *committed, int32_t *ar_argmax, int32_t *next_anchor)
+{
+    extern __shared__ int g[];
+    const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int i = warp; i < K; i += 8) {
+        const ArgPart *pp = parts + ((long long)b * K + i) * n_seg;
+        float bv = -INFINITY;
+        int bi = 0x7fffffff;
+        for (int s = lane; s < n_seg; s += 32) {
+            const ArgPart a = pp[s];
+            if (better(a.v, a.idx, bv, bi)) { bv = a.v; bi = a.idx; }
+        }
+#pragma unroll
+        for (int off = 16; off; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+            if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+        }
+        if (bi == 0x7fffffff) bi = 0;            // a row with no comparable value
+        if (lane == 0) { g[i] = bi; ar_argmax[(long long)b * K + i] = bi; }
+    }
+    __syncthreads();
+    __shared__ int n_sh;
+    if (threadIdx.x == 0) {
+        int m = 0;
+        while (m < K && draft[(long long)b * K + m] == g[m]) ++m;
+        const int n = m + 1 < K ? m + 1 : K;
+        n_sh = n;
+        n_commit[b] = n;
+        next_anchor[b] = g[n - 1];
+    }
+    __syncthreads();
+    const int n = n_sh;
+    for (int i = threadIdx.x; i < K; i += blockDim.x)
+        committed[(long long)b * K + i] = i < n ? g[i] : -1;
+}
+
 }  // namespace
+
+cudaError_t launch_consensus_finalize_wide(const ArgPart *parts, int n_seg, const int32_t *draft, int B,
+                                           int K, int32_t *n_commit, int32_t *committed,
+                                           int32_t *ar_argmax, int32_t *next_anchor, cudaStream_t st)
+{
+    consensus_finalize_wide_kernel<<<B, 256, K * sizeof(int), st>>>(parts, n_seg, draft, K, n_commit,
+                                                                     committed, ar_argmax, next_anchor);
+    count_launch();
+    return cudaGetLastError();
+}
 
 int consensus_segments(int B, int K, int V)
 {

@@ -1,0 +1,289 @@
+// Greedy tokens straight from the AR view's last hidden states: the LM-head product
+// logits[r][v] = hidden[r][:] . lm_head[v][:] on the 5th-generation tensor cores with the
+// per-row argmax of Eq. 8 taken in the accumulator read-out, so the [rows][vocab] logits
+// never reach memory.  bf16 operands, fp32 accumulation, the comparison on the fp32 sums.
+//
+// Tiling.  An item is (tile of 128 hidden rows, tile of 256 vocabulary entries); its product
+// runs over the hidden dimension in stages of 64 columns (one 128-byte swizzle panel: 16 KB
+// of hidden rows + 32 KB of LM-head rows per stage, four stages in flight).  A persistent
+// grid of one CTA per SM takes items round-robin with the row tile varying fastest, so the
+// CTAs that share a vocabulary tile read it at the same time and it crosses HBM once.  Rows
+// past the end of `hidden`, vocabulary entries past V and a ragged last stage are zero-filled
+// by the TMA unit; the read-out skips the padded vocabulary entries and never writes padded
+// rows.
+//
+// One CTA (192 threads, 193 KB of shared memory, all 512 TMEM columns = two accumulators):
+//   warp 0     producer: one lane issues the TMA loads of every stage
+//   warp 1     TMEM allocation and MMA issue (four 128x256x16 MMAs per stage) into
+//              accumulator (item & 1), so the product of the next item runs under the
+//              read-out of this one
+//   warps 2-5  read-out: thread = one row (TMEM lane); 256 fp32 sums are scanned in
+//              increasing vocabulary order with a strict '>' (the lowest id wins ties, a NaN
+//              never wins) and one (value, id) pair per (row, vocabulary tile) is stored.
+// The pairs are folded per row, and the accept rule applied, by the finalize kernel of the
+// logits-based consensus.
+//
+// Every mbarrier wait is bounded: on expiry the CTA records ORTHRUS_DEV_WAIT_TIMEOUT in the
+// status word, drains the copies it armed, frees its TMEM and returns.
+#include <mutex>
+#include <unordered_map>
+#include "common.cuh"
+#include "tc_ptx.cuh"
+
+namespace orthrus {
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int NSTAGE = 4;
+constexpr int NTHREADS = 192;
+constexpr int X_BYTES = BM * BK * 2, W_BYTES = BN * BK * 2, STAGE_BYTES = X_BYTES + W_BYTES;
+constexpr int OFF_BAR = NSTAGE * STAGE_BYTES;
+constexpr int OFF_MISC = OFF_BAR + 16 * 8;
+constexpr int SMEM_BYTES = OFF_MISC + 64;
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
+static_assert(2 * SMEM_BYTES > 228 * 1024, "one CTA per SM: it takes all 512 TMEM columns");
+enum { BAR_FULL = 0, BAR_EMPTY = NSTAGE, BAR_TFULL = 2 * NSTAGE, BAR_TEMPTY = BAR_TFULL + 2,
+       BAR_DONE = BAR_TEMPTY + 2, NUM_BARS };
+static_assert(NUM_BARS <= 16, "barrier area");
+constexpr uint32_t TM_COLS = 2 * BN;
+
+__device__ inline uint64_t policy_evict_last() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ inline uint64_t policy_evict_normal() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+struct HeadMaps { CUtensorMap x, w; };
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const int V, const int n_k,
+                      const int n_m, const int n_n, ArgPart *parts, int32_t *status)
+{
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const uint32_t sbase = smem_u32(smem);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + OFF_MISC + 8);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + OFF_MISC);
+    auto bar = [&](int i) { return sbase + OFF_BAR + i * 8; };
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_items = n_m * n_n;
+
+    if (tid == 0) *abort_flag = (sbase & 1023u) == 0 ? 0 : 1;   // swizzled tiles need 1 KB alignment
+    if (warp == 0 && lane == 0) {
+        for (int i = 0; i < 2 * NSTAGE; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(BAR_TFULL), 1); mbar_init(bar(BAR_TFULL + 1), 1);
+        mbar_init(bar(BAR_TEMPTY), 4); mbar_init(bar(BAR_TEMPTY + 1), 4);
+        mbar_init(bar(BAR_DONE), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+        prefetch_map(&tm.x); prefetch_map(&tm.w);
+    } else if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(TM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0 && !*abort_flag) {
+            const uint64_t pol_x = policy_evict_last();
+            // the LM head is read once when there is a single row tile
+            const uint64_t pol_w = n_m == 1 ? policy_evict_first() : policy_evict_normal();
+            int g = 0;
+            bool ok = true;
+            for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+                const int m = it % n_m, n = it / n_m;
+                for (int ks = 0; ks < n_k && ok; ++ks, ++g) {
+                    const int stage = g % NSTAGE, use = g / NSTAGE;
+                    if (use > 0) ok = mbar_wait(bar(BAR_EMPTY + stage), (use - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    const uint32_t dst = sbase + stage * STAGE_BYTES;
+                    mbar_expect_tx(bar(BAR_FULL + stage), STAGE_BYTES);
+                    tma_load_2d(dst, &tm.x, ks * BK, m * BM, bar(BAR_FULL + stage), pol_x);
+                    tma_load_2d(dst + X_BYTES, &tm.w, ks * BK, n * BN, bar(BAR_FULL + stage), pol_w);
+                }
+            }
+            if (*abort_flag) {
+                // give the copies that were armed a bounded time to land before smem is released
+                for (int j = max(0, g - NSTAGE); j < g; ++j) {
+                    int dummy = 0;
+                    mbar_wait(bar(BAR_FULL + j % NSTAGE), (j / NSTAGE) & 1, &dummy);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issue
+        constexpr uint32_t IDESC = make_idesc(BN, 0);           // both operands K-major
+        int g = 0, li = 0;
+        bool ok = !*abort_flag;
+        ok = __all_sync(0xffffffffu, ok);
+        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++li) {
+            const int buf = li & 1, buse = li >> 1;
+            if (buse > 0) ok = mbar_wait_warp(bar(BAR_TEMPTY + buf), (buse - 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            for (int ks = 0; ks < n_k && ok; ++ks, ++g) {
+                const int stage = g % NSTAGE, use = g / NSTAGE;
+                ok = mbar_wait_warp(bar(BAR_FULL + stage), use & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t x_addr = sbase + stage * STAGE_BYTES, w_addr = x_addr + X_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk)
+                        umma_ss(tmem + buf * BN, make_desc(x_addr + kk * 32, 16, 1024),
+                                make_desc(w_addr + kk * 32, 16, 1024), IDESC, (ks > 0) || (kk > 0));
+                    umma_commit(bar(BAR_EMPTY + stage));
+                }
+                __syncwarp();
+            }
+            if (ok && lane == 0) umma_commit(bar(BAR_TFULL + buf));
+            __syncwarp();
+        }
+        // every MMA issued so far must have retired before TMEM is freed
+        if (lane == 0) umma_commit(bar(BAR_DONE));
+        __syncwarp();
+        { int dummy = 0; mbar_wait_warp(bar(BAR_DONE), 0, &dummy); }
+        tc_fence_before();
+    } else {
+        // ------------------------------------------------------------------ read-out
+        const int quarter = warp & 3;                           // the TMEM lanes this warp may read
+        const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
+        int li = 0;
+        bool ok = !*abort_flag;
+        ok = __all_sync(0xffffffffu, ok);
+        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++li) {
+            const int m = it % n_m, n = it / n_m;
+            const int buf = li & 1, buse = li >> 1;
+            ok = mbar_wait_warp(bar(BAR_TFULL + buf), buse & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const int v0 = n * BN;
+            const int n_valid = min(BN, V - v0);
+            float best = -INFINITY;
+            int bidx = 0x7fffffff;
+#pragma unroll 1
+            for (int c = 0; c < BN; c += 64) {
+                uint32_t r[64];
+                tmem_ld32(lane_base + buf * BN + c, r);
+                tmem_ld32(lane_base + buf * BN + c + 32, r + 32);
+                tmem_ld_wait();
+                if (c + 64 <= n_valid) {
+#pragma unroll
+                    for (int j = 0; j < 64; ++j) {
+                        const float x = __uint_as_float(r[j]);
+                        if (x > best) { best = x; bidx = v0 + c + j; }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 64; ++j) {
+                        const float x = __uint_as_float(r[j]);
+                        if (c + j < n_valid && x > best) { best = x; bidx = v0 + c + j; }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_TEMPTY + buf));
+            const int row = m * BM + quarter * 32 + lane;
+            if (row < R) parts[(long long)row * n_n + n] = ArgPart{best, bidx};
+        }
+        tc_fence_before();
+    }
+
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TM_COLS) : "memory");
+    if (tid == 0 && *abort_flag && status) atomicOr(status, ORTHRUS_DEV_WAIT_TIMEOUT);
+}
+
+struct Map2Key {
+    const void *ptr; unsigned long long inner, outer; unsigned box_outer;
+    bool operator==(const Map2Key &o) const {
+        return ptr == o.ptr && inner == o.inner && outer == o.outer && box_outer == o.box_outer;
+    }
+};
+struct Map2KeyHash {
+    size_t operator()(const Map2Key &k) const {
+        size_t x = std::hash<const void *>()(k.ptr);
+        for (unsigned long long v : {k.inner, k.outer, (unsigned long long)k.box_outer})
+            x = (x ^ v) * 0x9E3779B97F4A7C15ull;
+        return x;
+    }
+};
+
+// A map over a row-major bf16 matrix [outer][inner]: boxes of 64 columns x box_outer rows,
+// 128-byte swizzle, zero fill outside the matrix.  Cached by (pointer, shape).
+bool get_map_2d(const void *ptr, unsigned long long inner, unsigned long long outer, unsigned box_outer,
+                CUtensorMap *out)
+{
+    static std::mutex mu;
+    static std::unordered_map<Map2Key, CUtensorMap, Map2KeyHash> cache;
+    std::lock_guard<std::mutex> lock(mu);
+    const Map2Key key{ptr, inner, outer, box_outer};
+    auto it = cache.find(key);
+    if (it != cache.end()) { *out = it->second; return true; }
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+    const cuuint64_t strides[1] = {(cuuint64_t)inner * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, box_outer};
+    const cuuint32_t estr[2] = {1, 1};
+    CUtensorMap tm;
+    const CUresult r = fn(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides,
+                          box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return false;
+    if (cache.size() > 1024) cache.clear();
+    cache.emplace(key, tm);
+    *out = tm;
+    return true;
+}
+
+}  // namespace
+
+int lm_head_vocab_tiles(int V) { return (V + BN - 1) / BN; }
+
+bool lm_head_supported() { return encode_fn() != nullptr; }
+
+// parts: [rows][vocab tiles] (value, id) pairs.  Returns cudaErrorNotSupported when the tensor
+// maps cannot be built.
+cudaError_t launch_lm_head_argmax(const void *hidden, const void *lm_head, int R, int V, int H,
+                                  ArgPart *parts, int32_t *status, cudaStream_t st)
+{
+    HeadMaps tm;
+    if (!get_map_2d(hidden, (unsigned long long)H, (unsigned long long)R, BM, &tm.x) ||
+        !get_map_2d(lm_head, (unsigned long long)H, (unsigned long long)V, BN, &tm.w))
+        return cudaErrorNotSupported;
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static bool configured[kMaxDevices] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+            e = cudaFuncSetAttribute(lm_head_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+            if (e != cudaSuccess) return e;
+            if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
+        }
+    }
+    const int n_m = (R + BM - 1) / BM, n_n = lm_head_vocab_tiles(V), n_k = (H + BK - 1) / BK;
+    const long long n_items = (long long)n_m * n_n;
+    const int grid = (int)(n_items < kNumSMs ? n_items : kNumSMs);
+    lm_head_argmax_kernel<<<grid, NTHREADS, SMEM_BYTES, st>>>(tm, R, V, n_k, n_m, n_n, parts, status);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace orthrus

@@ -88,3 +88,26 @@ def test_null_and_small_workspace(lib):
     assert a(ctypes.byref(L), None, 0x2000, 0x3000, 1, None, 0, None) == 1
     assert lib.lib().orthrus_set_path(b"bogus") == 1
     assert lib.lib().orthrus_set_path(b"auto") == 0
+
+
+def test_lm_head_consensus_rejects_misuse_before_launch(lib):
+    h = lib.lib().orthrus_lm_head_consensus
+    wsb = lib.lib().orthrus_lm_head_consensus_workspace_bytes
+    # one (value, id) pair per row and 256-entry vocabulary tile, after the header
+    assert wsb(2, 16, 1000) == 256 + 2 * 16 * 4 * 8
+    assert wsb(0, 16, 1000) == 0
+    ok = dict(hidden=0x1000, lm_head=0x2000, dtype=0, H=4096, draft=0x3000, B=1, K=16, V=151936,
+              n=0x4000, com=0x5000, arg=0x6000, nxt=0x7000, ws=0x8000, wsb=1 << 30)
+
+    def call(**kw):
+        a = dict(ok, **kw)
+        return h(a["hidden"], a["lm_head"], a["dtype"], a["H"], a["draft"], a["B"], a["K"], a["V"],
+                 a["n"], a["com"], a["arg"], a["nxt"], a["ws"], a["wsb"], None)
+
+    assert call(hidden=None) == 1 and call(lm_head=None) == 1 and call(ws=None) == 1
+    assert call(B=0) == 1 and call(H=0) == 1
+    assert call(dtype=1) == 2                      # fp32 operands are not supported
+    assert call(H=4100) == 2                       # rows must be a multiple of 16 bytes
+    assert call(hidden=0x1008) == 1                # 16-byte alignment of the operands
+    assert call(draft=0x3002) == 1
+    assert call(wsb=1024) == 4
