@@ -17,6 +17,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -34,6 +35,7 @@ from paper_2605_12825_b200 import workloads as W  # noqa: E402
 DEFAULT_WORKLOAD = "cfg2_8b_b1"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
+FALLBACK_BF16_TFLOPS = 1590.0
 
 
 # ----------------------------------------------------------------------------- helpers
@@ -45,6 +47,17 @@ def measured_peak():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+def measured_tensor_peak():
+    """(burst, sustained) dense bf16 TFLOP/s of the library GEMM measured on this machine."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return FALLBACK_BF16_TFLOPS, 1400.0, "fallback"
 
 
 # DRAM bytes (read + write) per launch of the attention kernel from the ncu capture summarised
@@ -438,12 +451,93 @@ def run_gpu(args):
                      "avg_launch_us": round(attend_ms * 1e3, 3),
                      "traffic": recorded_traffic(wl.name)},
     }
+    if args.lm_head > 0:
+        with torch.cuda.stream(stream):
+            out["lm_head_consensus"] = lm_head_measure(B, wl, args.lm_head, dev, stream,
+                                                       max(3, min(args.steps, 50)))
     if rank == 0:
         if not args.no_cpu_baseline and world == 1:
             out["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_budget, gpu_state=st)
         print(json.dumps(out), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def lm_head_measure(B, wl, hidden_dim, dev, stream, steps):
+    """Times the fused LM-head consensus (the step that feeds Eq. 8, with the logits kept on
+    chip) on the workload's (batch, block, vocab) and the given hidden size, and beside it the
+    two-step path it replaces: the library matrix product writing bf16 logits, then
+    orthrus_consensus_accept.  Operands are seeded device-side normals (timing only; parity
+    is the test suite's business).  The LM head is larger than L2 for every configuration."""
+    Bt, K, V, H = wl.batch, wl.block, wl.vocab, hidden_dim
+    g = torch.Generator(device=dev)
+    g.manual_seed(W.sub_seed(12825, wl.name, 0, "lm_head"))
+    hidden = torch.randn(Bt, K, H, device=dev, generator=g).to(torch.bfloat16)
+    lm_head = torch.empty(V, H, device=dev, dtype=torch.bfloat16)
+    for v0 in range(0, V, 16384):
+        v1 = min(V, v0 + 16384)
+        lm_head[v0:v1] = (torch.randn(v1 - v0, H, device=dev, generator=g) / math.sqrt(H)).to(torch.bfloat16)
+    draft = torch.randint(0, V, (Bt, K), device=dev, generator=g, dtype=torch.int32)
+    i32 = dict(dtype=torch.int32, device=dev)
+    outs = [torch.zeros(Bt, **i32), torch.zeros(Bt, K, **i32), torch.zeros(Bt, K, **i32), torch.zeros(Bt, **i32)]
+    outs2 = [torch.zeros_like(o) for o in outs]
+    ws = B.new_workspace(B.orthrus_lm_head_consensus_workspace_bytes(Bt, K, V), device=dev)
+    ws2 = B.new_workspace(B.orthrus_consensus_workspace_bytes(Bt, K, V), device=dev)
+    logits = torch.empty(Bt * K, V, device=dev, dtype=torch.bfloat16)
+    h2 = hidden.view(Bt * K, H)
+    w_t = lm_head.t()
+
+    def fused():
+        B.orthrus_lm_head_consensus(hidden, lm_head, draft, *outs, ws, stream=stream)
+
+    def two_step():
+        torch.matmul(h2, w_t, out=logits)
+        B.orthrus_consensus_accept(logits.view(Bt, K, V), draft, *outs2, ws2, stream=stream)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        stream.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        stream.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    n0 = B.orthrus_launch_count()
+    fused()
+    launches = B.orthrus_launch_count() - n0
+    ms_fused = timed(fused)
+    ms_two = timed(two_step)
+    status = B.orthrus_read_status(ws, stream)
+    if status != 0:
+        raise SystemExit(f"bench.py: device status word {status} after the LM-head measurement")
+    agree = float((outs[2] == outs2[2]).float().mean())
+    flops = 2.0 * Bt * K * V * H
+    nbytes = 2.0 * V * H + 2.0 * Bt * K * H
+    hbm, hbm_kind = measured_peak()
+    burst, sustained, tf_kind = measured_tensor_peak()
+    t_tensor, t_hbm = flops / (burst * 1e12), nbytes / (hbm * 1e9)
+    if t_tensor >= t_hbm:
+        roof = {"bound": "tensor", "achieved": round(flops / (ms_fused * 1e-3) / 1e12, 2), "peak": burst,
+                "peak_kind": tf_kind + " (library bf16 GEMM, burst)", "peak_sustained": sustained,
+                "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": round(nbytes / (ms_fused * 1e-3) / 1e9, 2), "peak": hbm,
+                "peak_kind": hbm_kind, "unit": "GB/s"}
+    roof["frac"] = round(roof["achieved"] / roof["peak"], 4)
+    roof["traffic"] = None
+    return {"hidden_dim": H, "rows": Bt * K, "vocab": V, "steps": steps,
+            "ms_fused": round(ms_fused, 5), "ms_two_step": round(ms_two, 5),
+            "two_step": "torch.matmul (library GEMM) writing bf16 logits + orthrus_consensus_accept",
+            "speedup_vs_two_step": round(ms_two / ms_fused, 3),
+            "tflops": round(flops / (ms_fused * 1e-3) / 1e12, 2),
+            "lm_head_gbs": round(nbytes / (ms_fused * 1e-3) / 1e9, 1),
+            "algorithmic_flops_per_call": flops, "algorithmic_bytes_per_call": nbytes,
+            "launches_per_call": launches, "greedy_tokens_equal_two_step": round(agree, 4),
+            "roofline": roof}
 
 
 # ----------------------------------------------------------------------------- oracle arm
@@ -574,6 +668,8 @@ def main():
                     help="> 0: the consensus phase uses rejection sampling instead of the greedy rule")
     ap.add_argument("--block", type=int, default=0,
                     help="override the block width K (the block-size sweep of Section 5)")
+    ap.add_argument("--lm-head", type=int, default=0, metavar="HIDDEN",
+                    help="also time the fused LM-head consensus at this hidden size (extra key)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-early-prefetch", action="store_true",
                     help="do not set ORTHRUS_LAYER_CACHE_QUIESCENT on the layers")

@@ -3,25 +3,30 @@
 // per-row argmax of Eq. 8 taken in the accumulator read-out, so the [rows][vocab] logits
 // never reach memory.  bf16 operands, fp32 accumulation, the comparison on the fp32 sums.
 //
-// Tiling.  An item is (tile of 128 hidden rows, tile of 256 vocabulary entries); its product
-// runs over the hidden dimension in stages of 64 columns (one 128-byte swizzle panel: 16 KB
-// of hidden rows + 32 KB of LM-head rows per stage, four stages in flight).  A persistent
-// grid of one CTA per SM takes items round-robin with the row tile varying fastest, so the
-// CTAs that share a vocabulary tile read it at the same time and it crosses HBM once.  Rows
-// past the end of `hidden`, vocabulary entries past V and a ragged last stage are zero-filled
-// by the TMA unit; the read-out skips the padded vocabulary entries and never writes padded
-// rows.
+// Tiling.  An item is (tile of BM hidden rows, tile of 256 vocabulary entries); its product
+// runs over the hidden dimension in stages of 64 columns (one 128-byte swizzle panel).  A
+// persistent grid of one CTA per SM takes items round-robin with the row tile varying
+// fastest, so the CTAs that share a vocabulary tile read it at the same time and it crosses
+// HBM once.  Rows past the end of `hidden`, vocabulary entries past V and a ragged last stage
+// are zero-filled by the TMA unit; the read-out skips the padded vocabulary entries and never
+// writes padded rows.
 //
-// One CTA (192 threads, 193 KB of shared memory, all 512 TMEM columns = two accumulators):
-//   warp 0     producer: one lane issues the TMA loads of every stage
-//   warp 1     TMEM allocation and MMA issue (four 128x256x16 MMAs per stage) into
-//              accumulator (item & 1), so the product of the next item runs under the
-//              read-out of this one
-//   warps 2-5  read-out: thread = one row (TMEM lane); 256 fp32 sums are scanned in
-//              increasing vocabulary order with a strict '>' (the lowest id wins ties, a NaN
-//              never wins) and one (value, id) pair per (row, vocabulary tile) is stored.
-// The pairs are folded per row, and the accept rule applied, by the finalize kernel of the
-// logits-based consensus.
+// Two shapes, both using all 512 TMEM columns as two 128 x 256 fp32 accumulators:
+//   MT = 1 (at most 128 rows: the LM head is streamed once and HBM binds).  BM = 128, four
+//          stages of 16 + 32 KB; the accumulators alternate between items, so the product of
+//          the next item runs under the read-out of this one.
+//   MT = 2 (more rows: the tensor pipe binds).  BM = 256, three stages of 32 + 32 KB; the two
+//          accumulators hold the two row halves of one item, which halves the bytes the SM
+//          pulls from L2 per MMA.  Within a stage the MMAs of the first half are issued
+//          first, so its read-out overlaps the last MMAs of the second half, and the read-out
+//          of the second half the first MMAs of the next item.
+//
+// One CTA: warp 0 producer (one lane issues the TMA loads of every stage), warp 1 TMEM
+// allocation and MMA issue (128x256x16 MMAs, four per accumulator and stage), then four
+// read-out warps per accumulator: thread = one row (TMEM lane); 256 fp32 sums are scanned in
+// increasing vocabulary order with a strict '>' (the lowest id wins ties, a NaN never wins)
+// and one (value, id) pair per (row, vocabulary tile) is stored.  The pairs are folded per
+// row, and the accept rule applied, by the finalize kernel of the logits-based consensus.
 //
 // Every mbarrier wait is bounded: on expiry the CTA records ORTHRUS_DEV_WAIT_TIMEOUT in the
 // status word, drains the copies it armed, frees its TMEM and returns.
@@ -33,18 +38,23 @@
 namespace orthrus {
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int NSTAGE = 4;
-constexpr int NTHREADS = 192;
-constexpr int X_BYTES = BM * BK * 2, W_BYTES = BN * BK * 2, STAGE_BYTES = X_BYTES + W_BYTES;
-constexpr int OFF_BAR = NSTAGE * STAGE_BYTES;
-constexpr int OFF_MISC = OFF_BAR + 16 * 8;
-constexpr int SMEM_BYTES = OFF_MISC + 64;
-static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
-static_assert(2 * SMEM_BYTES > 228 * 1024, "one CTA per SM: it takes all 512 TMEM columns");
-enum { BAR_FULL = 0, BAR_EMPTY = NSTAGE, BAR_TFULL = 2 * NSTAGE, BAR_TEMPTY = BAR_TFULL + 2,
-       BAR_DONE = BAR_TEMPTY + 2, NUM_BARS };
-static_assert(NUM_BARS <= 16, "barrier area");
+constexpr int BN = 256, BK = 64;
+constexpr int W_BYTES = BN * BK * 2, XSUB_BYTES = 128 * BK * 2;
+template <int MT> struct Shape {
+    static constexpr int BM = 128 * MT;
+    static constexpr int NSTAGE = MT == 1 ? 4 : 3;
+    static constexpr int NTHREADS = 64 + 128 * MT;
+    static constexpr int X_BYTES = MT * XSUB_BYTES;
+    static constexpr int STAGE_BYTES = X_BYTES + W_BYTES;
+    static constexpr int OFF_BAR = NSTAGE * STAGE_BYTES;
+    static constexpr int OFF_MISC = OFF_BAR + 16 * 8;
+    static constexpr int SMEM_BYTES = OFF_MISC + 64;
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
+    static_assert(2 * SMEM_BYTES > 228 * 1024, "one CTA per SM: it takes all 512 TMEM columns");
+    enum { BAR_FULL = 0, BAR_EMPTY = NSTAGE, BAR_TFULL = 2 * NSTAGE, BAR_TEMPTY = BAR_TFULL + 2,
+           BAR_DONE = BAR_TEMPTY + 2, NUM_BARS };
+    static_assert(NUM_BARS <= 16, "barrier area");
+};
 constexpr uint32_t TM_COLS = 2 * BN;
 
 __device__ inline uint64_t policy_evict_last() {
@@ -60,15 +70,20 @@ __device__ inline uint64_t policy_evict_normal() {
 
 struct HeadMaps { CUtensorMap x, w; };
 
-__global__ void __launch_bounds__(NTHREADS, 1)
+template <int MT>
+__global__ void __launch_bounds__(Shape<MT>::NTHREADS, 1)
 lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const int V, const int n_k,
                       const int n_m, const int n_n, ArgPart *parts, int32_t *status)
 {
+    using S = Shape<MT>;
+    constexpr int NSTAGE = S::NSTAGE, STAGE_BYTES = S::STAGE_BYTES, X_BYTES = S::X_BYTES, BM = S::BM;
+    constexpr int BAR_FULL = S::BAR_FULL, BAR_EMPTY = S::BAR_EMPTY, BAR_TFULL = S::BAR_TFULL,
+                  BAR_TEMPTY = S::BAR_TEMPTY, BAR_DONE = S::BAR_DONE;
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t sbase = smem_u32(smem);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + OFF_MISC + 8);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + OFF_MISC);
-    auto bar = [&](int i) { return sbase + OFF_BAR + i * 8; };
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + S::OFF_MISC + 8);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + S::OFF_MISC);
+    auto bar = [&](int i) { return sbase + S::OFF_BAR + i * 8; };
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_items = n_m * n_n;
 
@@ -90,6 +105,10 @@ lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const in
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+
+    // accumulator and its use count for row half `a` of this CTA's item number `li`
+    auto acc_of = [](int li, int a) { return MT == 1 ? (li & 1) : a; };
+    auto use_of = [](int li) { return MT == 1 ? (li >> 1) : li; };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
@@ -126,27 +145,32 @@ lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const in
         bool ok = !*abort_flag;
         ok = __all_sync(0xffffffffu, ok);
         for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++li) {
-            const int buf = li & 1, buse = li >> 1;
-            if (buse > 0) ok = mbar_wait_warp(bar(BAR_TEMPTY + buf), (buse - 1) & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
+            const int use = use_of(li);
             for (int ks = 0; ks < n_k && ok; ++ks, ++g) {
-                const int stage = g % NSTAGE, use = g / NSTAGE;
-                ok = mbar_wait_warp(bar(BAR_FULL + stage), use & 1, abort_flag);
+                const int stage = g % NSTAGE, suse = g / NSTAGE;
+                ok = mbar_wait_warp(bar(BAR_FULL + stage), suse & 1, abort_flag);
                 if (!ok) break;
-                tc_fence_after();
-                if (lane == 0) {
-                    const uint32_t x_addr = sbase + stage * STAGE_BYTES, w_addr = x_addr + X_BYTES;
+                const uint32_t x_addr = sbase + stage * STAGE_BYTES, w_addr = x_addr + X_BYTES;
 #pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk)
-                        umma_ss(tmem + buf * BN, make_desc(x_addr + kk * 32, 16, 1024),
-                                make_desc(w_addr + kk * 32, 16, 1024), IDESC, (ks > 0) || (kk > 0));
-                    umma_commit(bar(BAR_EMPTY + stage));
+                for (int a = 0; a < MT; ++a) {
+                    const int acc = acc_of(li, a);
+                    // the accumulator must have been read out before the item's first MMA clears it
+                    if (ks == 0 && use > 0) {
+                        ok = mbar_wait_warp(bar(BAR_TEMPTY + acc), (use - 1) & 1, abort_flag);
+                        if (!ok) break;
+                    }
+                    tc_fence_after();
+                    if (lane == 0) {
+#pragma unroll
+                        for (int kk = 0; kk < BK / 16; ++kk)
+                            umma_ss(tmem + acc * BN, make_desc(x_addr + a * XSUB_BYTES + kk * 32, 16, 1024),
+                                    make_desc(w_addr + kk * 32, 16, 1024), IDESC, (ks > 0) || (kk > 0));
+                        if (a == MT - 1) umma_commit(bar(BAR_EMPTY + stage));
+                        if (ks == n_k - 1) umma_commit(bar(BAR_TFULL + acc));
+                    }
+                    __syncwarp();
                 }
-                __syncwarp();
             }
-            if (ok && lane == 0) umma_commit(bar(BAR_TFULL + buf));
-            __syncwarp();
         }
         // every MMA issued so far must have retired before TMEM is freed
         if (lane == 0) umma_commit(bar(BAR_DONE));
@@ -156,14 +180,15 @@ lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const in
     } else {
         // ------------------------------------------------------------------ read-out
         const int quarter = warp & 3;                           // the TMEM lanes this warp may read
+        const int a = (warp - 2) >> 2;                          // row half (MT = 2)
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
         int li = 0;
         bool ok = !*abort_flag;
         ok = __all_sync(0xffffffffu, ok);
         for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++li) {
             const int m = it % n_m, n = it / n_m;
-            const int buf = li & 1, buse = li >> 1;
-            ok = mbar_wait_warp(bar(BAR_TFULL + buf), buse & 1, abort_flag);
+            const int acc = acc_of(li, a), use = use_of(li);
+            ok = mbar_wait_warp(bar(BAR_TFULL + acc), use & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
             const int v0 = n * BN;
@@ -173,8 +198,8 @@ lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const in
 #pragma unroll 1
             for (int c = 0; c < BN; c += 64) {
                 uint32_t r[64];
-                tmem_ld32(lane_base + buf * BN + c, r);
-                tmem_ld32(lane_base + buf * BN + c + 32, r + 32);
+                tmem_ld32(lane_base + acc * BN + c, r);
+                tmem_ld32(lane_base + acc * BN + c + 32, r + 32);
                 tmem_ld_wait();
                 if (c + 64 <= n_valid) {
 #pragma unroll
@@ -192,8 +217,8 @@ lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const in
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_TEMPTY + buf));
-            const int row = m * BM + quarter * 32 + lane;
+            if (lane == 0) mbar_arrive(bar(BAR_TEMPTY + acc));
+            const int row = m * BM + a * 128 + quarter * 32 + lane;
             if (row < R) parts[(long long)row * n_n + n] = ArgPart{best, bidx};
         }
         tc_fence_before();
@@ -249,6 +274,33 @@ bool get_map_2d(const void *ptr, unsigned long long inner, unsigned long long ou
     return true;
 }
 
+template <int MT>
+cudaError_t launch_shape(const HeadMaps &tm, int R, int V, int H, ArgPart *parts, int32_t *status, cudaStream_t st)
+{
+    using S = Shape<MT>;
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static bool configured[kMaxDevices] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
+            e = cudaFuncSetAttribute(lm_head_argmax_kernel<MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     S::SMEM_BYTES);
+            if (e != cudaSuccess) return e;
+            if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
+        }
+    }
+    const int n_m = (R + S::BM - 1) / S::BM, n_n = lm_head_vocab_tiles(V), n_k = (H + BK - 1) / BK;
+    const long long n_items = (long long)n_m * n_n;
+    const int grid = (int)(n_items < kNumSMs ? n_items : kNumSMs);
+    lm_head_argmax_kernel<MT><<<grid, S::NTHREADS, S::SMEM_BYTES, st>>>(tm, R, V, n_k, n_m, n_n, parts, status);
+    count_launch();
+    return cudaGetLastError();
+}
+
 }  // namespace
 
 int lm_head_vocab_tiles(int V) { return (V + BN - 1) / BN; }
@@ -260,30 +312,13 @@ bool lm_head_supported() { return encode_fn() != nullptr; }
 cudaError_t launch_lm_head_argmax(const void *hidden, const void *lm_head, int R, int V, int H,
                                   ArgPart *parts, int32_t *status, cudaStream_t st)
 {
+    const int mt = R > 128 ? 2 : 1;
     HeadMaps tm;
-    if (!get_map_2d(hidden, (unsigned long long)H, (unsigned long long)R, BM, &tm.x) ||
+    if (!get_map_2d(hidden, (unsigned long long)H, (unsigned long long)R, 128 * mt, &tm.x) ||
         !get_map_2d(lm_head, (unsigned long long)H, (unsigned long long)V, BN, &tm.w))
         return cudaErrorNotSupported;
-    constexpr int kMaxDevices = 64;
-    static std::mutex mu;
-    static bool configured[kMaxDevices] = {};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    {
-        std::lock_guard<std::mutex> lock(mu);
-        if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
-            e = cudaFuncSetAttribute(lm_head_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-            if (e != cudaSuccess) return e;
-            if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
-        }
-    }
-    const int n_m = (R + BM - 1) / BM, n_n = lm_head_vocab_tiles(V), n_k = (H + BK - 1) / BK;
-    const long long n_items = (long long)n_m * n_n;
-    const int grid = (int)(n_items < kNumSMs ? n_items : kNumSMs);
-    lm_head_argmax_kernel<<<grid, NTHREADS, SMEM_BYTES, st>>>(tm, R, V, n_k, n_m, n_n, parts, status);
-    count_launch();
-    return cudaGetLastError();
+    return mt == 2 ? launch_shape<2>(tm, R, V, H, parts, status, st)
+                   : launch_shape<1>(tm, R, V, H, parts, status, st);
 }
 
 }  // namespace orthrus

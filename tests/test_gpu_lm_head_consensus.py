@@ -148,3 +148,36 @@ def test_repeated_calls_and_unfused_path_agree_on_clear_rows():
     clear = ((top2[:, 0] - top2[:, 1]) > 2.0 ** -7 * top2[:, 0].abs().clamp(min=1.0)).reshape(B, K)
     assert int(clear.sum()) > B * K // 2
     assert torch.equal(outs[2].cpu()[clear], first[2][clear])
+
+
+def test_full_size_serving_shape_on_sampled_rows():
+    """The ragged serving configuration at full size (32 sequences x 32 positions, hidden
+    4096, vocabulary 128256: eight row tiles, 501 vocabulary tiles, 4008 items on the
+    persistent grid).  The oracle computes sampled rows one by one; integer outputs are
+    checked against the accept rule on the kernel's own tokens for every sequence."""
+    B, K, V, H = 32, 32, 128256, 4096
+    hidden, lm_head = rand_case(B, K, V, H, seed=12825)
+    rows = torch.tensor([0, 127, 128, 500, 1023, 777], dtype=torch.int32)   # tile edges and interiors
+    ref_arg, top2 = oracle.lm_head_argmax(hidden.reshape(B * K, H), lm_head, rows)
+    g = torch.Generator().manual_seed(2)
+    draft = torch.randint(0, V, (B, K), generator=g, dtype=torch.int32)
+    for j, r in enumerate(rows.tolist()):
+        draft[r // K, r % K] = ref_arg[j]
+    n, com, arg, nxt = run_fused(hidden, lm_head, draft)
+    flat = arg.reshape(-1)
+    for j, r in enumerate(rows.tolist()):
+        scale = max(1.0, abs(float(top2[j, 0])))
+        if float(top2[j, 0] - top2[j, 1]) > TOL * scale:
+            assert int(flat[r]) == int(ref_arg[j]), r
+        else:
+            got = float(hidden.reshape(B * K, H)[r].double() @ lm_head[int(flat[r])].double())
+            assert got >= float(top2[j, 0]) - TOL * scale
+    assert bool(((arg >= 0) & (arg < V)).all())
+    rn, rcom, rnxt = oracle.accept_rule(arg.contiguous(), draft)
+    assert torch.equal(n, rn) and torch.equal(com, rcom) and torch.equal(nxt, rnxt)
+    # every row's token must at least beat a random sample of other ids on the device
+    hd, wd = hidden.cuda().reshape(B * K, H).float(), lm_head.cuda()
+    cand = torch.randint(0, V, (64,), generator=g)
+    lg_c = hd @ wd[cand.cuda()].float().T
+    lg_a = (hd * wd[flat.cuda().long()].float()).sum(-1)
+    assert bool((lg_a.unsqueeze(1) >= lg_c - 1e-3).all())
