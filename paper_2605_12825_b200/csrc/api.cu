@@ -337,7 +337,7 @@ orthrus_status_t orthrus_consensus_accept_static(const void *ar_logits, int32_t 
 size_t orthrus_lm_head_consensus_workspace_bytes(int32_t batch, int32_t block, int32_t vocab)
 {
     if (batch < 1 || block < 1 || vocab < 1) return 0;
-    return kHeaderBytes + (size_t)batch * block * lm_head_vocab_tiles(vocab) * sizeof(ArgPart);
+    return kHeaderBytes + (size_t)batch * block * lm_head_max_vocab_tiles(vocab) * sizeof(ArgPart);
 }
 
 orthrus_status_t orthrus_lm_head_consensus(const void *hidden, const void *lm_head, int32_t dtype,
@@ -365,7 +365,7 @@ orthrus_status_t orthrus_lm_head_consensus(const void *hidden, const void *lm_he
                                           static_cast<int32_t *>(workspace), st);
     if (e == cudaErrorNotSupported) return ORTHRUS_ERR_UNSUPPORTED;
     if (e == cudaSuccess)
-        e = launch_consensus_finalize_wide(parts, lm_head_vocab_tiles(vocab), draft, batch, block, n_commit,
+        e = launch_consensus_finalize_wide(parts, lm_head_vocab_tiles(batch * block, vocab), draft, batch, block, n_commit,
                                            committed, ar_argmax, next_anchor, st);
     return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
 }

@@ -70,7 +70,8 @@ struct ArgPart { float v; int idx; };    // the best (value, id) of one stretch 
 cudaError_t launch_consensus_finalize_wide(const ArgPart *parts, int n_seg, const int32_t *draft, int B,
                                            int K, int32_t *n_commit, int32_t *committed,
                                            int32_t *ar_argmax, int32_t *next_anchor, cudaStream_t st);
-int lm_head_vocab_tiles(int V);
+int lm_head_vocab_tiles(int R, int V);     // (value, id) pairs per row for R rows, vocabulary V
+int lm_head_max_vocab_tiles(int V);        // the most any row count needs
 bool lm_head_supported();
 cudaError_t launch_lm_head_argmax(const void *hidden, const void *lm_head, int R, int V, int H,
                                   ArgPart *parts, int32_t *status, cudaStream_t st);

@@ -3,7 +3,8 @@
 // per-row argmax of Eq. 8 taken in the accumulator read-out, so the [rows][vocab] logits
 // never reach memory.  bf16 operands, fp32 accumulation, the comparison on the fp32 sums.
 //
-// Tiling.  An item is (tile of BM hidden rows, tile of 256 vocabulary entries); its product
+// Tiling.  An item is (tile of BM hidden rows, tile of bn <= 256 vocabulary entries, bn chosen
+// by the host so that the items fill whole waves of the grid); its product
 // runs over the hidden dimension in stages of 64 columns (one 128-byte swizzle panel).  A
 // persistent grid of one CTA per SM takes items round-robin with the row tile varying
 // fastest, so the CTAs that share a vocabulary tile read it at the same time and it crosses
@@ -73,7 +74,7 @@ struct HeadMaps { CUtensorMap x, w; };
 template <int MT>
 __global__ void __launch_bounds__(Shape<MT>::NTHREADS, 1)
 lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const int V, const int n_k,
-                      const int n_m, const int n_n, ArgPart *parts, int32_t *status)
+                      const int n_m, const int n_n, const int bn, ArgPart *parts, int32_t *status)
 {
     using S = Shape<MT>;
     constexpr int NSTAGE = S::NSTAGE, STAGE_BYTES = S::STAGE_BYTES, X_BYTES = S::X_BYTES, BM = S::BM;
@@ -125,9 +126,9 @@ lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const in
                     if (use > 0) ok = mbar_wait(bar(BAR_EMPTY + stage), (use - 1) & 1, abort_flag);
                     if (!ok) break;
                     const uint32_t dst = sbase + stage * STAGE_BYTES;
-                    mbar_expect_tx(bar(BAR_FULL + stage), STAGE_BYTES);
+                    mbar_expect_tx(bar(BAR_FULL + stage), (uint32_t)(X_BYTES + bn * BK * 2));
                     tma_load_2d(dst, &tm.x, ks * BK, m * BM, bar(BAR_FULL + stage), pol_x);
-                    tma_load_2d(dst + X_BYTES, &tm.w, ks * BK, n * BN, bar(BAR_FULL + stage), pol_w);
+                    tma_load_2d(dst + X_BYTES, &tm.w, ks * BK, n * bn, bar(BAR_FULL + stage), pol_w);
                 }
             }
             if (*abort_flag) {
@@ -140,7 +141,7 @@ lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const in
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issue
-        constexpr uint32_t IDESC = make_idesc(BN, 0);           // both operands K-major
+        const uint32_t IDESC = make_idesc((uint32_t)bn, 0);     // both operands K-major
         int g = 0, li = 0;
         bool ok = !*abort_flag;
         ok = __all_sync(0xffffffffu, ok);
@@ -191,12 +192,12 @@ lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const in
             ok = mbar_wait_warp(bar(BAR_TFULL + acc), use & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            const int v0 = n * BN;
-            const int n_valid = min(BN, V - v0);
+            const int v0 = n * bn;
+            const int n_valid = min(bn, V - v0);                // columns past it hold nothing of this item
             float best = -INFINITY;
             int bidx = 0x7fffffff;
 #pragma unroll 1
-            for (int c = 0; c < BN; c += 64) {
+            for (int c = 0; c < n_valid; c += 64) {
                 uint32_t r[64];
                 tmem_ld32(lane_base + acc * BN + c, r);
                 tmem_ld32(lane_base + acc * BN + c + 32, r + 32);
@@ -275,7 +276,8 @@ bool get_map_2d(const void *ptr, unsigned long long inner, unsigned long long ou
 }
 
 template <int MT>
-cudaError_t launch_shape(const HeadMaps &tm, int R, int V, int H, ArgPart *parts, int32_t *status, cudaStream_t st)
+cudaError_t launch_shape(const HeadMaps &tm, int R, int V, int H, int bn, ArgPart *parts, int32_t *status,
+                         cudaStream_t st)
 {
     using S = Shape<MT>;
     constexpr int kMaxDevices = 64;
@@ -293,32 +295,54 @@ cudaError_t launch_shape(const HeadMaps &tm, int R, int V, int H, ArgPart *parts
             if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
         }
     }
-    const int n_m = (R + S::BM - 1) / S::BM, n_n = lm_head_vocab_tiles(V), n_k = (H + BK - 1) / BK;
+    const int n_m = (R + S::BM - 1) / S::BM, n_n = (V + bn - 1) / bn, n_k = (H + BK - 1) / BK;
     const long long n_items = (long long)n_m * n_n;
     const int grid = (int)(n_items < kNumSMs ? n_items : kNumSMs);
-    lm_head_argmax_kernel<MT><<<grid, S::NTHREADS, S::SMEM_BYTES, st>>>(tm, R, V, n_k, n_m, n_n, parts, status);
+    lm_head_argmax_kernel<MT><<<grid, S::NTHREADS, S::SMEM_BYTES, st>>>(tm, R, V, n_k, n_m, n_n, bn, parts,
+                                                                       status);
     count_launch();
     return cudaGetLastError();
 }
 
 }  // namespace
 
-int lm_head_vocab_tiles(int V) { return (V + BN - 1) / BN; }
+// Width of the vocabulary tiles (a multiple of 16 from 128 to 256, the N of the MMAs): the one
+// whose item count fills the persistent grid's waves best.  The busiest CTA works through
+// waves x (width + a per-item overhead worth about 16 columns); ties go to the wider tile,
+// which re-reads the hidden rows less often.
+int lm_head_tile_width(int R, int V)
+{
+    const int n_m = R > 128 ? (R + 255) / 256 : 1;
+    int best_bn = BN;
+    long long best_cost = -1;
+    for (int bn = BN; bn >= 128; bn -= 16) {
+        const long long items = (long long)n_m * ((V + bn - 1) / bn);
+        const long long waves = (items + kNumSMs - 1) / kNumSMs;
+        const long long cost = waves * (bn + 16);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_bn = bn; }
+    }
+    return best_bn;
+}
+
+int lm_head_vocab_tiles(int R, int V) { const int bn = lm_head_tile_width(R, V); return (V + bn - 1) / bn; }
+
+int lm_head_max_vocab_tiles(int V) { return (V + 127) / 128; }
 
 bool lm_head_supported() { return encode_fn() != nullptr; }
 
-// parts: [rows][vocab tiles] (value, id) pairs.  Returns cudaErrorNotSupported when the tensor
-// maps cannot be built.
+// parts: [rows][lm_head_vocab_tiles(R, V)] (value, id) pairs.  Returns cudaErrorNotSupported when
+// the tensor maps cannot be built.
 cudaError_t launch_lm_head_argmax(const void *hidden, const void *lm_head, int R, int V, int H,
                                   ArgPart *parts, int32_t *status, cudaStream_t st)
 {
     const int mt = R > 128 ? 2 : 1;
+    const int bn = lm_head_tile_width(R, V);
     HeadMaps tm;
     if (!get_map_2d(hidden, (unsigned long long)H, (unsigned long long)R, 128 * mt, &tm.x) ||
-        !get_map_2d(lm_head, (unsigned long long)H, (unsigned long long)V, BN, &tm.w))
+        !get_map_2d(lm_head, (unsigned long long)H, (unsigned long long)V, bn, &tm.w))
         return cudaErrorNotSupported;
-    return mt == 2 ? launch_shape<2>(tm, R, V, H, parts, status, st)
-                   : launch_shape<1>(tm, R, V, H, parts, status, st);
+    return mt == 2 ? launch_shape<2>(tm, R, V, H, bn, parts, status, st)
+                   : launch_shape<1>(tm, R, V, H, bn, parts, status, st);
 }
 
 }  // namespace orthrus

@@ -93,8 +93,8 @@ def test_null_and_small_workspace(lib):
 def test_lm_head_consensus_rejects_misuse_before_launch(lib):
     h = lib.lib().orthrus_lm_head_consensus
     wsb = lib.lib().orthrus_lm_head_consensus_workspace_bytes
-    # one (value, id) pair per row and 256-entry vocabulary tile, after the header
-    assert wsb(2, 16, 1000) == 256 + 2 * 16 * 4 * 8
+    # one (value, id) pair per row and vocabulary tile (at least 128 entries wide), after the header
+    assert wsb(2, 16, 1000) == 256 + 2 * 16 * 8 * 8
     assert wsb(0, 16, 1000) == 0
     ok = dict(hidden=0x1000, lm_head=0x2000, dtype=0, H=4096, draft=0x3000, B=1, K=16, V=151936,
               n=0x4000, com=0x5000, arg=0x6000, nxt=0x7000, ws=0x8000, wsb=1 << 30)
