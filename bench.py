@@ -60,24 +60,40 @@ def measured_tensor_peak():
         return FALLBACK_BF16_TFLOPS, 1400.0, "fallback"
 
 
-# DRAM bytes (read + write) per launch of the attention kernel from the ncu capture summarised
-# in profiles/attend_tc_cfg2_8b_b1.md, with the first 16 hex digits of the SHA-256 of the
-# kernel source the capture was taken from: once that file changes the figure is stale.
-NCU_TRAFFIC = {"cfg2_8b_b1": (17048320, "5022ee0e01cd465d")}
+# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/, each
+# with the first 16 hex digits of the SHA-256 of the kernel sources the capture was taken
+# from: once those files change the figure is stale and None is reported.
+NCU_TRAFFIC = {"cfg2_8b_b1": (17048320, "debb11c45e119c74")}
+NCU_TRAFFIC_SOURCES = ("attend_tc.cu", "tc_ptx.cuh")
+NCU_TRAFFIC_LM_HEAD = {("cfg2_8b_b1", 4096): (1249298400, "44372c8e30c2919c"),
+                       ("cfg3_ragged", 4096): (1066727528, "44372c8e30c2919c")}
+NCU_TRAFFIC_LM_HEAD_SOURCES = ("lm_head_argmax.cu", "tc_ptx.cuh")
+
+
+def _source_digest(names):
+    import hashlib
+    m = hashlib.sha256()
+    try:
+        for n in names:
+            with open(os.path.join(ROOT, "paper_2605_12825_b200", "csrc", n), "rb") as f:
+                m.update(f.read())
+    except OSError:
+        return None
+    return m.hexdigest()[:16]
 
 
 def recorded_traffic(workload: str):
     rec = NCU_TRAFFIC.get(workload)
     if rec is None:
         return None
-    import hashlib
-    path = os.path.join(ROOT, "paper_2605_12825_b200", "csrc", "attend_tc.cu")
-    try:
-        with open(path, "rb") as f:
-            digest = hashlib.sha256(f.read()).hexdigest()[:16]
-    except OSError:
+    return rec[0] if _source_digest(NCU_TRAFFIC_SOURCES) == rec[1] else None
+
+
+def recorded_lm_head_traffic(workload: str, hidden_dim: int):
+    rec = NCU_TRAFFIC_LM_HEAD.get((workload, hidden_dim))
+    if rec is None:
         return None
-    return rec[0] if digest == rec[1] else None
+    return rec[0] if _source_digest(NCU_TRAFFIC_LM_HEAD_SOURCES) == rec[1] else None
 
 
 def attend_bytes(wl: W.Workload, lens) -> int:
@@ -528,7 +544,7 @@ def lm_head_measure(B, wl, hidden_dim, dev, stream, steps):
         roof = {"bound": "hbm", "achieved": round(nbytes / (ms_fused * 1e-3) / 1e9, 2), "peak": hbm,
                 "peak_kind": hbm_kind, "unit": "GB/s"}
     roof["frac"] = round(roof["achieved"] / roof["peak"], 4)
-    roof["traffic"] = None
+    roof["traffic"] = recorded_lm_head_traffic(wl.name, H)
     return {"hidden_dim": H, "rows": Bt * K, "vocab": V, "steps": steps,
             "ms_fused": round(ms_fused, 5), "ms_two_step": round(ms_two, 5),
             "two_step": "torch.matmul (library GEMM) writing bf16 logits + orthrus_consensus_accept",
