@@ -3,7 +3,7 @@
 Test harness only.  Everything off the hot path (embeddings, RMSNorm, RoPE, the Q/K/V/O
 projections of both views, the SwiGLU FFN, the LM head) is plain torch; the four steps of
 the hot path go through the C ABI: orthrus_diffusion_block_attend, orthrus_ar_verify_attend,
-orthrus_consensus_accept and orthrus_kv_append_layers.  Only the diffusion view's Q/K/V
+orthrus_consensus_accept (or orthrus_lm_head_consensus) and orthrus_kv_append_layers.  Only the diffusion view's Q/K/V
 projections are separate weights; output projection, FFN, norms, embeddings and LM head are
 shared with the AR view (Section 3.1).  The block is the anchor followed by K-1 copies of a
 mask embedding (Section 3.3); block position i has rotary position P_b + i.
@@ -98,9 +98,10 @@ class Decoder:
         return prompt[:, -1].to(torch.int32)
 
     # ------------------------------------------------------------------ one pass through the layers
-    def forward_block(self, tokens, view, block):
+    def forward_block(self, tokens, view, block, return_hidden=False):
         """tokens [B][block] (id == vocab selects the mask embedding).  view 'diff' or 'ar'.
-        Returns (logits [B][block][V], per-layer block K, per-layer block V)."""
+        Returns (logits [B][block][V], per-layer block K, per-layer block V), with
+        return_hidden also the final-norm hidden states [B][block][H] the LM head is applied to."""
         b = self.b
         B = tokens.shape[0]
         h = self.emb[tokens.long()]
@@ -124,8 +125,17 @@ class Decoder:
             h = h + out.view(B, block, self.Hq * self.d) @ lw["wo"]
             h = self.ffn(lw, h)
             ks.append(k); vs.append(v)
-        logits = (self.norm(h) @ self.lm_head).contiguous()
+        hn = self.norm(h).contiguous()
+        logits = (hn @ self.lm_head).contiguous()
+        if return_hidden:
+            return logits, ks, vs, hn
         return logits, ks, vs
+
+    def lm_head_rows(self):
+        """The LM head as [V][H] rows, the layout orthrus_lm_head_consensus takes."""
+        if not hasattr(self, "_lm_head_rows"):
+            self._lm_head_rows = self.lm_head.t().contiguous()
+        return self._lm_head_rows
 
     def commit(self, ks, vs, n_commit, block):
         self.b.orthrus_kv_append_layers(self.layer_objs(block), ks, vs, n_commit, True, self.ws)

@@ -19,8 +19,9 @@ from _gpu_util import binding
 pytestmark = pytest.mark.gpu
 
 
-def greedy_trajectory(dec, anchor, n_new):
-    """Width-1 decoding with the AR view: returns tokens [B][n_new] and top-2 gaps."""
+def greedy_trajectory(dec, anchor, n_new, fused=False):
+    """Width-1 decoding with the AR view: returns tokens [B][n_new] and top-2 gaps.  fused:
+    the greedy token comes from orthrus_lm_head_consensus on the hidden states."""
     b = dec.b
     B = anchor.shape[0]
     i32 = dict(dtype=torch.int32, device="cuda")
@@ -28,9 +29,14 @@ def greedy_trajectory(dec, anchor, n_new):
     cws = b.new_workspace(b.orthrus_consensus_workspace_bytes(B, 1, dec.V))
     toks, gaps = [], []
     draft = torch.zeros(B, 1, **i32)
+    if fused:
+        cws = b.new_workspace(b.orthrus_lm_head_consensus_workspace_bytes(B, 1, dec.V))
     for _ in range(n_new):
-        logits, ks, vs = dec.forward_block(anchor.view(B, 1), "ar", 1)
-        b.orthrus_consensus_accept(logits, draft, *outs, cws)
+        logits, ks, vs, hn = dec.forward_block(anchor.view(B, 1), "ar", 1, return_hidden=True)
+        if fused:
+            b.orthrus_lm_head_consensus(hn, dec.lm_head_rows(), draft, *outs, cws)
+        else:
+            b.orthrus_consensus_accept(logits, draft, *outs, cws)
         top2 = logits.float().topk(2, dim=-1).values[:, 0]
         gaps.append((top2[:, 0] - top2[:, 1]).cpu())
         dec.commit(ks, vs, outs[0], 1)
@@ -39,7 +45,7 @@ def greedy_trajectory(dec, anchor, n_new):
     return torch.stack(toks, 1), torch.stack(gaps, 1)
 
 
-def run_loop(dtype, layers, hidden, n_q, n_kv, d, ffn, vocab, B, T, K, n_new, rate, eps):
+def run_loop(dtype, layers, hidden, n_q, n_kv, d, ffn, vocab, B, T, K, n_new, rate, eps, fused=False):
     b = binding()
     b.orthrus_set_path("auto")
     cap = T + n_new + 2 * K + 8
@@ -48,7 +54,7 @@ def run_loop(dtype, layers, hidden, n_q, n_kv, d, ffn, vocab, B, T, K, n_new, ra
 
     ref = Decoder(b, layers, hidden, n_q, n_kv, d, ffn, vocab, dtype, B, cap, K, seed=3)
     anchor0 = ref.prefill(prompt)
-    traj, gaps = greedy_trajectory(ref, anchor0, n_new + K)
+    traj, gaps = greedy_trajectory(ref, anchor0, n_new + K, fused)
 
     dec = Decoder(b, layers, hidden, n_q, n_kv, d, ffn, vocab, dtype, B, cap, K, seed=3,
                   flags=b.LAYER_CACHE_QUIESCENT)
@@ -56,6 +62,7 @@ def run_loop(dtype, layers, hidden, n_q, n_kv, d, ffn, vocab, B, T, K, n_new, ra
     assert torch.equal(anchor.cpu(), anchor0.cpu())
     streams = [[] for _ in range(B)]
     cycles, total = 0, 0
+    fws = b.new_workspace(b.orthrus_lm_head_consensus_workspace_bytes(B, K, vocab)) if fused else None
     while min(len(s) for s in streams) < n_new:
         done = torch.tensor([len(s) for s in streams])
         # forced drafts: the trajectory token with probability `rate`, else a uniform token
@@ -72,10 +79,23 @@ def run_loop(dtype, layers, hidden, n_q, n_kv, d, ffn, vocab, B, T, K, n_new, ra
         assert torch.isfinite(d_logits.float()).all()
         # forward pass 2: the AR view over [anchor, draft_1 .. draft_{K-1}]
         ar_in = torch.cat([anchor.view(B, 1), draft[:, :K - 1]], dim=1)
-        logits, ks, vs = dec.forward_block(ar_in, "ar", K)
-        b.orthrus_consensus_accept(logits, draft, dec.n_commit, dec.committed, dec.ar_argmax,
-                                   dec.next_anchor, dec.cws)
-        rn, rcom, rarg, rnxt = oracle.consensus_accept(logits.cpu(), draft.cpu())
+        logits, ks, vs, hn = dec.forward_block(ar_in, "ar", K, return_hidden=True)
+        if fused:
+            # the greedy tokens straight from the hidden states; the oracle's fp64 logits decide
+            # wherever its two largest are clearly apart, and the accept rule is exact
+            b.orthrus_lm_head_consensus(hn, dec.lm_head_rows(), draft, dec.n_commit, dec.committed,
+                                        dec.ar_argmax, dec.next_anchor, fws)
+            assert b.orthrus_read_status(fws) == 0
+            oarg, top2 = oracle.lm_head_argmax(hn.cpu().reshape(B * K, -1), dec.lm_head_rows().cpu())
+            clear = ((top2[:, 0] - top2[:, 1]) > 1e-4 * top2[:, 0].abs().clamp(min=1.0)).reshape(B, K)
+            garg = dec.ar_argmax.cpu()
+            assert torch.equal(garg[clear], oarg.reshape(B, K)[clear])
+            rn, rcom, rnxt = oracle.accept_rule(garg.contiguous(), draft.cpu())
+            rarg = garg
+        else:
+            b.orthrus_consensus_accept(logits, draft, dec.n_commit, dec.committed, dec.ar_argmax,
+                                       dec.next_anchor, dec.cws)
+            rn, rcom, rarg, rnxt = oracle.consensus_accept(logits.cpu(), draft.cpu())
         assert torch.equal(dec.n_commit.cpu(), rn) and torch.equal(dec.committed.cpu(), rcom)
         assert torch.equal(dec.ar_argmax.cpu(), rarg) and torch.equal(dec.next_anchor.cpu(), rnxt)
         assert int(rn.min()) >= 1 and int(rn.max()) <= K
@@ -114,6 +134,16 @@ def test_generation_bf16_tcgen05_shapes():
     assert ties <= 2
     assert 1.5 < mean_n < 4.5
     assert binding().orthrus_last_path() == "tcgen05"
+
+
+def test_generation_bf16_consensus_fused_with_the_lm_head():
+    """The same loop with the greedy tokens taken straight from the last hidden states
+    (orthrus_lm_head_consensus): no logits tensor is handed to the consensus, in the loop or in
+    the width-1 reference run."""
+    mean_n, ties = run_loop(torch.bfloat16, layers=3, hidden=512, n_q=8, n_kv=2, d=128, ffn=1024,
+                            vocab=2000, B=4, T=300, K=16, n_new=48, rate=0.65, eps=0.25, fused=True)
+    assert ties <= 2
+    assert 1.5 < mean_n < 4.5
 
 
 def test_sampled_generation_loop_fp32():
