@@ -31,6 +31,7 @@
 //
 // Every mbarrier wait is bounded: on expiry the CTA records ORTHRUS_DEV_WAIT_TIMEOUT in the
 // status word, drains the copies it armed, frees its TMEM and returns.
+#include <cstdlib>
 #include <mutex>
 #include <unordered_map>
 #include "common.cuh"
@@ -70,6 +71,35 @@ __device__ inline uint64_t policy_evict_normal() {
 }
 
 struct HeadMaps { CUtensorMap x, w; };
+
+// Read-out of one accumulator row: this thread's TMEM lane, columns [0, n_valid) from column
+// address `taddr`, scanned in increasing order with a strict '>' (the lowest id wins ties, a
+// NaN never wins).  Nothing compares greater than -inf: then idx stays 0x7fffffff.
+__device__ inline void scan_accumulator(uint32_t taddr, int n_valid, int v0, float &best, int &bidx)
+{
+    best = -INFINITY;
+    bidx = 0x7fffffff;
+#pragma unroll 1
+    for (int c = 0; c < n_valid; c += 64) {
+        uint32_t r[64];
+        tmem_ld32(taddr + c, r);
+        tmem_ld32(taddr + c + 32, r + 32);
+        tmem_ld_wait();
+        if (c + 64 <= n_valid) {
+#pragma unroll
+            for (int j = 0; j < 64; ++j) {
+                const float x = __uint_as_float(r[j]);
+                if (x > best) { best = x; bidx = v0 + c + j; }
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 64; ++j) {
+                const float x = __uint_as_float(r[j]);
+                if (c + j < n_valid && x > best) { best = x; bidx = v0 + c + j; }
+            }
+        }
+    }
+}
 
 template <int MT>
 __global__ void __launch_bounds__(Shape<MT>::NTHREADS, 1)
@@ -194,28 +224,9 @@ lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const in
             tc_fence_after();
             const int v0 = n * bn;
             const int n_valid = min(bn, V - v0);                // columns past it hold nothing of this item
-            float best = -INFINITY;
-            int bidx = 0x7fffffff;
-#pragma unroll 1
-            for (int c = 0; c < n_valid; c += 64) {
-                uint32_t r[64];
-                tmem_ld32(lane_base + acc * BN + c, r);
-                tmem_ld32(lane_base + acc * BN + c + 32, r + 32);
-                tmem_ld_wait();
-                if (c + 64 <= n_valid) {
-#pragma unroll
-                    for (int j = 0; j < 64; ++j) {
-                        const float x = __uint_as_float(r[j]);
-                        if (x > best) { best = x; bidx = v0 + c + j; }
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 64; ++j) {
-                        const float x = __uint_as_float(r[j]);
-                        if (c + j < n_valid && x > best) { best = x; bidx = v0 + c + j; }
-                    }
-                }
-            }
+            float best;
+            int bidx;
+            scan_accumulator(lane_base + acc * BN, n_valid, v0, best, bidx);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_TEMPTY + acc));
@@ -229,6 +240,216 @@ lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const in
     tc_fence_after();
     if (warp == 1)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TM_COLS) : "memory");
+    if (tid == 0 && *abort_flag && status) atomicOr(status, ORTHRUS_DEV_WAIT_TIMEOUT);
+}
+
+// ---------------------------------------------------------------------------- two-SM shape
+//
+// Opt-in (ORTHRUS_LM_HEAD_PAIR=1) for more than 128 rows: the two CTAs of a cluster share
+// every item of 256 rows x bn vocabulary entries through one MMA of M = 256
+// (tcgen05.mma.cta_group::2, issued by the leader, CTA rank 0).  Each CTA stages its own 128
+// hidden rows and its own half of the LM-head tile (bn / 2 rows), so an SM loads and reads
+// from shared memory two thirds of what the one-SM 256-row shape needs per flop, and keeps its
+// two accumulators for alternate items, so the read-out is hidden.  Stages are 128 hidden
+// columns wide (two swizzle panels per operand, 64 KB per CTA, three stages): with 64-column
+// stages the per-stage barrier round and commits were measured to cost a quarter of the time.
+// Each CTA reads its 128 result rows out of its own TMEM.
+//
+// Barriers (same offsets in both CTAs): both producers' loads complete on the leader's FULL
+// barrier; the leader's MMA warp commits to the EMPTY and TFULL barriers of both CTAs with
+// one multicast commit; the read-out warps of both CTAs arrive on the leader's TEMPTY barrier.
+// The loads name no multicast.
+//
+// Measured on the serving shape (1024 x 128256 x 4096) it equals the one-SM 256-row shape
+// (735 against 732 us): both run at the power cap, so the one-SM shape stays the default.
+namespace pair {
+constexpr int NSTAGE = 3;
+constexpr int NTHREADS = 192;
+constexpr int KPANELS = 2;                             // 64-column panels per stage
+constexpr int WPANEL_BYTES = W_BYTES / 2;              // up to 128 LM-head rows x 64 columns
+constexpr int X_BYTES = KPANELS * XSUB_BYTES;          // 128 rows of hidden x 128 columns
+constexpr int STAGE_BYTES = X_BYTES + KPANELS * WPANEL_BYTES;
+constexpr int OFF_BAR = NSTAGE * STAGE_BYTES;
+constexpr int OFF_MISC = OFF_BAR + 24 * 8;
+constexpr int SMEM_BYTES = OFF_MISC + 64;
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
+static_assert(2 * SMEM_BYTES > 228 * 1024, "one CTA per SM: it takes all 512 TMEM columns");
+enum { BAR_FULL = 0, BAR_EMPTY = NSTAGE, BAR_TFULL = 2 * NSTAGE, BAR_TEMPTY = BAR_TFULL + 2,
+       BAR_DONE = BAR_TEMPTY + 2, NUM_BARS };
+static_assert(NUM_BARS <= 24, "barrier area");
+}  // namespace pair
+
+// D[tmem of both CTAs] (+)= A . B with M = 256 over the CTA pair
+__device__ inline void umma_ss_pair(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+                 " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+// arrival on a barrier of either CTA (cluster-window address) once the pair's MMAs so far retire
+__device__ inline void umma_commit_pair(uint32_t bar_cluster) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(bar_cluster) : "memory");
+}
+// tile load into this CTA's shared memory whose bytes are counted on a barrier of either CTA
+__device__ inline void tma_load_2d_pair(uint32_t dst, const CUtensorMap *tm, int c0, int c1, uint32_t bar_cluster,
+                                        uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+                 " [%0], [%1, {%2, %3}], [%4], %5;"
+                 ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar_cluster), "l"(policy) : "memory");
+}
+// the same arrival on the barrier at this offset in both CTAs of the pair
+__device__ inline void umma_commit_both(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+__device__ inline void mbar_arrive_cluster(uint32_t bar_cluster) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+// instruction descriptor as make_idesc, for M = 256 over the pair
+__host__ __device__ constexpr uint32_t make_idesc_pair(uint32_t n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((256u >> 4) << 24);
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(pair::NTHREADS, 1)
+lm_head_argmax_pair_kernel(const __grid_constant__ HeadMaps tm, const int R, const int V, const int n_k,
+                           const int n_m, const int n_n, const int bn, ArgPart *parts, int32_t *status)
+{
+    using namespace pair;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const uint32_t sbase = smem_u32(smem);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + OFF_MISC + 8);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + OFF_MISC);
+    auto bar = [&](int i) { return sbase + OFF_BAR + i * 8; };
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int rank = (int)cluster_rank();                       // 0: leader
+    const int n_clusters = gridDim.x >> 1, cluster_id = blockIdx.x >> 1;
+    const int n_items = n_m * n_n;
+    const int half = bn >> 1;                                   // LM-head rows per CTA and item
+
+    if (tid == 0) *abort_flag = (sbase & 1023u) == 0 ? 0 : 1;   // swizzled tiles need 1 KB alignment
+    if (warp == 0 && lane == 0) {
+        for (int i = 0; i < 2 * NSTAGE; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(BAR_TFULL), 1); mbar_init(bar(BAR_TFULL + 1), 1);
+        mbar_init(bar(BAR_TEMPTY), 8); mbar_init(bar(BAR_TEMPTY + 1), 8);   // 4 warps of each CTA
+        mbar_init(bar(BAR_DONE), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+        prefetch_map(&tm.x); prefetch_map(&tm.w);
+    } else if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(TM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                       // the peer's barriers exist before anything signals them
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer (both CTAs)
+        if (lane == 0 && !*abort_flag) {
+            const uint64_t pol_x = policy_evict_last();
+            const uint64_t pol_w = n_m == 1 ? policy_evict_first() : policy_evict_normal();
+            const uint32_t stage_tx = 2u * KPANELS * (uint32_t)(XSUB_BYTES + half * BK * 2);   // both CTAs' bytes
+            int g = 0;
+            bool ok = true;
+            for (int it = cluster_id; it < n_items && ok; it += n_clusters) {
+                const int m = it % n_m, n = it / n_m;
+                for (int ks = 0; ks < n_k && ok; ++ks, ++g) {
+                    const int stage = g % NSTAGE, use = g / NSTAGE;
+                    if (use > 0) ok = mbar_wait(bar(BAR_EMPTY + stage), (use - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    const uint32_t dst = sbase + stage * STAGE_BYTES;
+                    const uint32_t full = map_to_rank(bar(BAR_FULL + stage), 0);
+                    if (rank == 0) mbar_expect_tx(bar(BAR_FULL + stage), stage_tx);
+#pragma unroll
+                    for (int pnl = 0; pnl < KPANELS; ++pnl) {
+                        const int col = (ks * KPANELS + pnl) * BK;   // past H: zero-filled
+                        tma_load_2d_pair(dst + pnl * XSUB_BYTES, &tm.x, col, m * 256 + rank * 128, full, pol_x);
+                        tma_load_2d_pair(dst + X_BYTES + pnl * WPANEL_BYTES, &tm.w, col, n * bn + rank * half,
+                                         full, pol_w);
+                    }
+                }
+            }
+            if (*abort_flag && rank == 0) {
+                // give the copies that were armed a bounded time to land before smem is released
+                for (int j = max(0, g - NSTAGE); j < g; ++j) {
+                    int dummy = 0;
+                    mbar_wait(bar(BAR_FULL + j % NSTAGE), (j / NSTAGE) & 1, &dummy);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issue (leader)
+        if (rank == 0) {
+            const uint32_t IDESC = make_idesc_pair((uint32_t)bn);
+            int g = 0, li = 0;
+            bool ok = !*abort_flag;
+            ok = __all_sync(0xffffffffu, ok);
+            for (int it = cluster_id; it < n_items && ok; it += n_clusters, ++li) {
+                const int buf = li & 1, buse = li >> 1;
+                if (buse > 0) ok = mbar_wait_warp(bar(BAR_TEMPTY + buf), (buse - 1) & 1, abort_flag);
+                if (!ok) break;
+                for (int ks = 0; ks < n_k && ok; ++ks, ++g) {
+                    const int stage = g % NSTAGE, use = g / NSTAGE;
+                    ok = mbar_wait_warp(bar(BAR_FULL + stage), use & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t x_addr = sbase + stage * STAGE_BYTES, w_addr = x_addr + X_BYTES;
+#pragma unroll
+                        for (int kk = 0; kk < KPANELS * BK / 16; ++kk)
+                            umma_ss_pair(tmem + buf * BN,
+                                         make_desc(x_addr + (kk >> 2) * XSUB_BYTES + (kk & 3) * 32, 16, 1024),
+                                         make_desc(w_addr + (kk >> 2) * WPANEL_BYTES + (kk & 3) * 32, 16, 1024),
+                                         IDESC, (ks > 0) || (kk > 0));
+                        umma_commit_both(bar(BAR_EMPTY + stage));
+                        if (ks == n_k - 1) umma_commit_both(bar(BAR_TFULL + buf));
+                    }
+                    __syncwarp();
+                }
+            }
+            // every MMA issued so far must have retired before TMEM is freed
+            if (lane == 0) umma_commit_pair(bar(BAR_DONE));
+            __syncwarp();
+            { int dummy = 0; mbar_wait_warp(bar(BAR_DONE), 0, &dummy); }
+        }
+        tc_fence_before();
+    } else {
+        // ------------------------------------------------------------------ read-out (both CTAs)
+        const int quarter = warp & 3;                           // the TMEM lanes this warp may read
+        const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
+        int li = 0;
+        bool ok = !*abort_flag;
+        ok = __all_sync(0xffffffffu, ok);
+        for (int it = cluster_id; it < n_items && ok; it += n_clusters, ++li) {
+            const int m = it % n_m, n = it / n_m;
+            const int buf = li & 1, buse = li >> 1;
+            ok = mbar_wait_warp(bar(BAR_TFULL + buf), buse & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const int v0 = n * bn;
+            const int n_valid = min(bn, V - v0);
+            float best;
+            int bidx;
+            scan_accumulator(lane_base + buf * BN, n_valid, v0, best, bidx);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_rank(bar(BAR_TEMPTY + buf), 0));
+            const int row = m * 256 + rank * 128 + quarter * 32 + lane;
+            if (row < R) parts[(long long)row * n_n + n] = ArgPart{best, bidx};
+        }
+        tc_fence_before();
+    }
+
+    // neither CTA may leave, or free its TMEM, while the other can still signal its barriers or
+    // the leader's MMAs can still write its TMEM
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TM_COLS) : "memory");
     if (tid == 0 && *abort_flag && status) atomicOr(status, ORTHRUS_DEV_WAIT_TIMEOUT);
 }
 
@@ -304,27 +525,88 @@ cudaError_t launch_shape(const HeadMaps &tm, int R, int V, int H, int bn, ArgPar
     return cudaGetLastError();
 }
 
+// Clusters of two CTAs of the pair kernel the current device can keep resident (0: not asked
+// for with ORTHRUS_LM_HEAD_PAIR=1, none, or the query failed); looked up once per device.
+int pair_clusters()
+{
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static int cached[kMaxDevices];
+    static bool known[kMaxDevices] = {};
+    static const bool enabled = [] { const char *e = getenv("ORTHRUS_LM_HEAD_PAIR"); return e && atoi(e) == 1; }();
+    if (!enabled) return 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    std::lock_guard<std::mutex> lock(mu);
+    if (known[dev]) return cached[dev];
+    int n = 0;
+    if (cudaFuncSetAttribute(lm_head_argmax_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             pair::SMEM_BYTES) == cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * kNumSMs, 1, 1);
+        cfg.blockDim = dim3(pair::NTHREADS);
+        cfg.dynamicSmemBytes = pair::SMEM_BYTES;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        if (cudaOccupancyMaxActiveClusters(&n, lm_head_argmax_pair_kernel, &cfg) != cudaSuccess) n = 0;
+    }
+    (void)cudaGetLastError();
+    if (n > kNumSMs / 2) n = kNumSMs / 2;
+    cached[dev] = n; known[dev] = true;
+    return n;
+}
+
+cudaError_t launch_pair(const HeadMaps &tm, int R, int V, int H, int bn, int clusters, ArgPart *parts,
+                        int32_t *status, cudaStream_t st)
+{
+    const int n_m = (R + 255) / 256, n_n = (V + bn - 1) / bn;
+    const int n_k = (H + pair::KPANELS * BK - 1) / (pair::KPANELS * BK);
+    const long long n_items = (long long)n_m * n_n;
+    const int n_cl = (int)(n_items < clusters ? n_items : clusters);
+    lm_head_argmax_pair_kernel<<<2 * n_cl, pair::NTHREADS, pair::SMEM_BYTES, st>>>(tm, R, V, n_k, n_m, n_n, bn,
+                                                                                  parts, status);
+    count_launch();
+    return cudaGetLastError();
+}
+
 }  // namespace
 
-// Width of the vocabulary tiles (a multiple of 16 from 128 to 256, the N of the MMAs): the one
-// whose item count fills the persistent grid's waves best.  The busiest CTA works through
+// Width of the vocabulary tiles (the N of the MMAs, from 128 to 256): the one whose item count
+// fills the waves of the persistent grid best.  The busiest CTA (or CTA pair) works through
 // waves x (width + a per-item overhead worth about 16 columns); ties go to the wider tile,
-// which re-reads the hidden rows less often.
-int lm_head_tile_width(int R, int V)
+// which re-reads the hidden rows less often.  `pairs` > 0: the two-SM shape on that many
+// clusters, widths in multiples of 32 (each CTA holds half a tile).
+static int tile_width(int R, int V, int pairs)
 {
     const int n_m = R > 128 ? (R + 255) / 256 : 1;
+    const int workers = pairs > 0 ? pairs : kNumSMs, step = pairs > 0 ? 32 : 16;
     int best_bn = BN;
     long long best_cost = -1;
-    for (int bn = BN; bn >= 128; bn -= 16) {
+    for (int bn = BN; bn >= 128; bn -= step) {
         const long long items = (long long)n_m * ((V + bn - 1) / bn);
-        const long long waves = (items + kNumSMs - 1) / kNumSMs;
+        const long long waves = (items + workers - 1) / workers;
         const long long cost = waves * (bn + 16);
         if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_bn = bn; }
     }
     return best_bn;
 }
 
-int lm_head_vocab_tiles(int R, int V) { const int bn = lm_head_tile_width(R, V); return (V + bn - 1) / bn; }
+// the shape a problem runs in on the current device: clusters of the two-SM shape (0: one-SM
+// shapes) and the tile width
+static void plan(int R, int V, int *pairs, int *bn)
+{
+    *pairs = R > 128 ? pair_clusters() : 0;
+    *bn = tile_width(R, V, *pairs);
+}
+
+int lm_head_vocab_tiles(int R, int V)
+{
+    int pairs, bn;
+    plan(R, V, &pairs, &bn);
+    return (V + bn - 1) / bn;
+}
 
 int lm_head_max_vocab_tiles(int V) { return (V + 127) / 128; }
 
@@ -335,12 +617,14 @@ bool lm_head_supported() { return encode_fn() != nullptr; }
 cudaError_t launch_lm_head_argmax(const void *hidden, const void *lm_head, int R, int V, int H,
                                   ArgPart *parts, int32_t *status, cudaStream_t st)
 {
+    int pairs, bn;
+    plan(R, V, &pairs, &bn);
     const int mt = R > 128 ? 2 : 1;
-    const int bn = lm_head_tile_width(R, V);
     HeadMaps tm;
-    if (!get_map_2d(hidden, (unsigned long long)H, (unsigned long long)R, 128 * mt, &tm.x) ||
-        !get_map_2d(lm_head, (unsigned long long)H, (unsigned long long)V, bn, &tm.w))
+    if (!get_map_2d(hidden, (unsigned long long)H, (unsigned long long)R, pairs > 0 ? 128 : 128 * mt, &tm.x) ||
+        !get_map_2d(lm_head, (unsigned long long)H, (unsigned long long)V, pairs > 0 ? bn / 2 : bn, &tm.w))
         return cudaErrorNotSupported;
+    if (pairs > 0) return launch_pair(tm, R, V, H, bn, pairs, parts, status, st);
     return mt == 2 ? launch_shape<2>(tm, R, V, H, bn, parts, status, st)
                    : launch_shape<1>(tm, R, V, H, bn, parts, status, st);
 }
