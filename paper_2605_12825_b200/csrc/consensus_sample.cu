@@ -17,6 +17,7 @@
 // Exponentials are fp32; every sum is carried in double and taken in a fixed order, and
 // references are integers so that rescaling is exact: the result is reproducible run to run
 // and departs from an exact evaluation only by the rounding of the individual exponentials.
+#include <cstdlib>
 #include "common.cuh"
 
 namespace orthrus {
@@ -115,14 +116,20 @@ template <typename T> __host__ __device__ inline bool vector_ok(const void *base
 struct StatPart { float ma, md; double sa, sd; };       // per (row, segment)
 struct Sum2 { double x, y; };                           // (residual mass, AR mass) of a segment
 
-// 1. per (row, segment): (reference, sum) of both logit rows, in the log2 domain scaled by c = log2(e) / T
+// 1. per (row, segment): (reference, sum) of both logit rows, in the log2 domain scaled by c = log2(e) / T.
+// The launch covers block positions [k0, k1) of every sequence; with `fail` given, sequences
+// whose first rejection is already known (fail[b] < K) are skipped: verification halts at the
+// first rejected draft, so their later rows are never looked at.
 template <typename T>
 __global__ void __launch_bounds__(kThreads) sample_stats_kernel(const T *la, const T *ld, int V, int seg_len,
-                                                                float c, StatPart *parts, int vec)
+                                                                float c, StatPart *parts, int vec, int K, int k0,
+                                                                int k1, const int *fail)
 {
     constexpr int N = Elem<T>::N;
     __shared__ RefSum sh[kThreads / 32];
-    const int row = blockIdx.y, seg = blockIdx.x;
+    const int seq = blockIdx.y / (k1 - k0), seg = blockIdx.x;
+    if (fail != nullptr && fail[seq] < K) return;
+    const int row = seq * K + k0 + blockIdx.y % (k1 - k0);
     const int start = seg * seg_len, end = min(V, start + seg_len);
     const T *ra = la + (long long)row * V, *rd = ld + (long long)row * V;
     RefSum a{-INFINITY, 0.0}, d{-INFINITY, 0.0};
@@ -160,17 +167,21 @@ struct RowStat { float ma, md; double inv_za, inv_zd; int row; int pad; };   // 
 
 // 2. per sequence: fold the segments, take the accept tests, find the first failure
 template <typename T>
+// for block positions [k0, k1); fail[b] carries the outcome between the stages (K: no rejection
+// so far).  A sequence's results are written by the stage that settles it: the one that finds
+// its first rejection, or the last one.
 __global__ void sample_decide_kernel(const T *la, const T *ld, const StatPart *parts, int n_seg, int K, int V,
                                      float c, const int32_t *draft, const float *u_accept,
                                      int32_t *n_commit, int32_t *committed, int32_t *next_anchor,
-                                     RowStat *stat)
+                                     RowStat *stat, int k0, int k1, int *fail)
 {
     extern __shared__ StatPart folded[];        // [K]
     __shared__ int first_fail;
     const int b = blockIdx.x;
+    if (k0 > 0 && fail[b] < K) return;          // settled by an earlier stage
     if (threadIdx.x == 0) first_fail = K;
     __syncthreads();
-    for (int i = threadIdx.x; i < K; i += blockDim.x) {
+    for (int i = k0 + threadIdx.x; i < k1; i += blockDim.x) {
         const long long row = (long long)b * K + i;
         RefSum a{-INFINITY, 0.0}, d{-INFINITY, 0.0};
         for (int s = 0; s < n_seg; ++s) {
@@ -186,7 +197,9 @@ __global__ void sample_decide_kernel(const T *la, const T *ld, const StatPart *p
         if (!((double)u_accept[row] * qy <= py)) atomicMin(&first_fail, i);
     }
     __syncthreads();
-    const int j = first_fail;                   // K: every draft kept
+    const int j = first_fail;                   // K: every draft so far kept
+    if (threadIdx.x == 0) fail[b] = j;
+    if (j >= K && k1 < K) return;               // still open: the next stage goes on
     const int n = j < K ? j + 1 : K;
     for (int i = threadIdx.x; i < K; i += blockDim.x)
         committed[(long long)b * K + i] = i < min(j, K) ? draft[(long long)b * K + i] : -1;
@@ -194,7 +207,7 @@ __global__ void sample_decide_kernel(const T *la, const T *ld, const StatPart *p
         n_commit[b] = n;
         RowStat st;
         st.row = j < K ? j : -1;
-        const StatPart f = folded[j < K ? j : 0];
+        const StatPart f = j < K ? folded[j] : StatPart{0.f, 0.f, 1.0, 1.0};
         st.ma = f.ma; st.inv_za = 1.0 / f.sa; st.md = f.md; st.inv_zd = 1.0 / f.sd;
         st.pad = 0;
         stat[b] = st;
@@ -336,7 +349,23 @@ int sample_pick_segments(int V) { return (V + kPickSegMax - 1) / kPickSegMax; }
 size_t sample_workspace_bytes(int B, int K, int V)
 {
     return (size_t)B * K * sample_stat_segments(B, K, V) * sizeof(StatPart) + (size_t)B * sizeof(RowStat) +
-           (size_t)B * sample_pick_segments(V) * sizeof(Sum2);
+           (size_t)B * sample_pick_segments(V) * sizeof(Sum2) + (size_t)B * sizeof(int);
+}
+
+// Block positions verified by the first statistics pass.  Verification halts at the first
+// rejected draft, so rows behind it need not be looked at: when the two logit tensors are
+// large enough for the pass to be bound by throughput, the first pass covers a quarter of the
+// block (at least 4 positions) and a second pass the rest, for the sequences still open only.
+// More stages were measured slower (each costs two dependent launches), and small problems
+// are bound by launch latency and take one pass.  ORTHRUS_SAMPLE_FIRST_STAGE overrides.
+int sample_first_stage(int B, int K, int V)
+{
+    const long long bytes = 2LL * B * K * V * 2;
+    static const int forced = [] { const char *e = getenv("ORTHRUS_SAMPLE_FIRST_STAGE"); return e ? atoi(e) : 0; }();
+    if (forced > 0) return forced < K ? forced : K;
+    if (K <= 4 || bytes < (64LL << 20)) return K;
+    const int k1 = (K + 3) / 4;
+    return k1 < 4 ? 4 : k1;
 }
 
 template <typename T>
@@ -354,22 +383,31 @@ static cudaError_t launch_sample_t(const void *ar_logits, const void *diff_logit
     const int vec = vector_ok<T>(la, V) && vector_ok<T>(ld, V);
     StatPart *parts = reinterpret_cast<StatPart *>(ws);
     RowStat *stat = reinterpret_cast<RowStat *>(ws + (size_t)B * K * n_seg * sizeof(StatPart));
-    Sum2 *seg_sums = reinterpret_cast<Sum2 *>(reinterpret_cast<unsigned char *>(stat) + (size_t)B * sizeof(RowStat));
-    sample_stats_kernel<T><<<dim3(n_seg, B * K), kThreads, 0, st>>>(la, ld, V, seg_len, c, parts, vec);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    const int threads = K <= 32 ? 32 : ((K + 31) / 32 * 32 > 256 ? 256 : (K + 31) / 32 * 32);
-    sample_decide_kernel<T><<<B, threads, K * sizeof(StatPart), st>>>(la, ld, parts, n_seg, K, V, c, draft, u_accept,
-                                                                  n_commit, committed, next_anchor, stat);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
     const int n_seg2 = sample_pick_segments(V);
+    Sum2 *seg_sums = reinterpret_cast<Sum2 *>(reinterpret_cast<unsigned char *>(stat) + (size_t)B * sizeof(RowStat));
+    int *fail = reinterpret_cast<int *>(reinterpret_cast<unsigned char *>(seg_sums) + (size_t)B * n_seg2 * sizeof(Sum2));
+    const int threads = K <= 32 ? 32 : ((K + 31) / 32 * 32 > 256 ? 256 : (K + 31) / 32 * 32);
+    const int k_first = sample_first_stage(B, K, V);
+    cudaError_t e = cudaSuccess;
+    int launches = 2;
+    for (int k0 = 0, k1 = k_first; k0 < K; k0 = k1, k1 = K) {
+        sample_stats_kernel<T><<<dim3(n_seg, B * (k1 - k0)), kThreads, 0, st>>>(la, ld, V, seg_len, c, parts, vec, K,
+                                                                               k0, k1, k0 > 0 ? fail : nullptr);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        sample_decide_kernel<T><<<B, threads, K * sizeof(StatPart), st>>>(la, ld, parts, n_seg, K, V, c, draft,
+                                                                      u_accept, n_commit, committed, next_anchor,
+                                                                      stat, k0, k1, fail);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        launches += 2;
+    }
     sample_residual_kernel<T><<<dim3(n_seg2, B), kThreads, 0, st>>>(la, ld, K, V, kPickSegMax, c, stat, seg_sums);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     sample_pick_kernel<T><<<B, kThreads, 0, st>>>(la, ld, K, V, kPickSegMax, n_seg2, c, stat, seg_sums, u_resample,
                                                   committed, next_anchor);
-    count_launch(4);
+    count_launch(launches);
     return cudaGetLastError();
 }
 

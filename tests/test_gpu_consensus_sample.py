@@ -133,3 +133,19 @@ def test_rejects_bad_arguments_on_the_host():
     null = list(args); null[1] = None
     assert f(*null) == 1
     assert b.orthrus_launch_count() == n0
+
+
+def test_staged_verification_in_a_child_process():
+    """Large problems verify the block in two stages (the second only for sequences without a
+    rejection so far).  The stage boundary is chosen when the library is first used, so the
+    small cases above are repeated in a child process with the boundary forced to 2 positions:
+    rejections before, at and after the boundary, and blocks kept whole."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, ORTHRUS_SAMPLE_FIRST_STAGE="2")
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.abspath(__file__), "-x", "-q",
+                        "-k", "matches_oracle or temperatures or every_draft_kept or distribution"],
+                       env=env, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
+    assert " passed" in r.stdout
