@@ -234,6 +234,9 @@ orthrus_status_t orthrus_consensus_accept_static(const void *ar_logits, int32_t 
  * header initialised by orthrus_workspace_init; a wait inside the kernel that does not end
  * reports ORTHRUS_DEV_WAIT_TIMEOUT through orthrus_read_status and leaves the outputs of
  * that call undefined.  Two launches; nothing is allocated and the stream is not synchronised.
+ * The first call on each device sets kernel attributes and builds the tensor maps of its
+ * operands (cached by pointer and shape): make that call outside of any stream capture; later
+ * calls with the same buffers can be captured into a CUDA graph.
  */
 size_t orthrus_lm_head_consensus_workspace_bytes(int32_t batch, int32_t block, int32_t vocab);
 orthrus_status_t orthrus_lm_head_consensus(const void *hidden, const void *lm_head, int32_t dtype,

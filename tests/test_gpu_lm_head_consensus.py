@@ -181,3 +181,37 @@ def test_full_size_serving_shape_on_sampled_rows():
     lg_c = hd @ wd[cand.cuda()].float().T
     lg_a = (hd * wd[flat.cuda().long()].float()).sum(-1)
     assert bool((lg_a.unsqueeze(1) >= lg_c - 1e-3).all())
+
+
+def test_replay_from_a_cuda_graph_follows_new_inputs():
+    """The call allocates nothing and never synchronises, so (after one eager call has set the
+    kernel attributes) it can be captured; a replay must see the buffers' current contents."""
+    b = binding()
+    B, K, V, H = 2, 16, 3000, 256
+    hidden, lm_head = rand_case(B, K, V, H, seed=5)
+    hd, wd = hidden.cuda(), lm_head.cuda()
+    ws = b.new_workspace(b.orthrus_lm_head_consensus_workspace_bytes(B, K, V))
+    i32 = dict(dtype=torch.int32, device="cuda")
+    draft = torch.zeros(B, K, **i32)
+    outs = [torch.zeros(B, **i32), torch.zeros(B, K, **i32), torch.zeros(B, K, **i32), torch.zeros(B, **i32)]
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        b.orthrus_lm_head_consensus(hd, wd, draft, *outs, ws, stream=stream)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            b.orthrus_lm_head_consensus(hd, wd, draft, *outs, ws, stream=stream)
+        for seed in (6, 7):
+            h2, _ = rand_case(B, K, V, H, seed=seed)
+            ref_arg, top2 = oracle.lm_head_argmax(h2.reshape(B * K, H), lm_head)
+            d2 = drafts_from(ref_arg.reshape(B, K), V, 0.7, torch.Generator().manual_seed(seed))
+            hd.copy_(h2.cuda()); draft.copy_(d2.cuda())
+            g.replay()
+            stream.synchronize()
+            arg = outs[2].cpu()
+            clear = ((top2[:, 0] - top2[:, 1]) > TOL * top2[:, 0].abs().clamp(min=1.0)).reshape(B, K)
+            assert torch.equal(arg[clear], ref_arg.reshape(B, K)[clear])
+            rn, rcom, rnxt = oracle.accept_rule(arg.contiguous(), d2)
+            assert torch.equal(outs[0].cpu(), rn) and torch.equal(outs[1].cpu(), rcom)
+            assert torch.equal(outs[3].cpu(), rnxt)
+    assert b.orthrus_read_status(ws) == 0
