@@ -12,13 +12,14 @@
 // are zero-filled by the TMA unit; the read-out skips the padded vocabulary entries and never
 // writes padded rows.
 //
-// Two shapes, both using all 512 TMEM columns as two 128 x 256 fp32 accumulators:
+// Two one-SM shapes (and an optional two-SM one, further down), all using the 512 TMEM columns
+// as two 128 x 256 fp32 accumulators:
 //   MT = 1 (at most 128 rows: the LM head is streamed once and HBM binds).  BM = 128, four
 //          stages of 16 + 32 KB; the accumulators alternate between items, so the product of
 //          the next item runs under the read-out of this one.
 //   MT = 2 (more rows: the tensor pipe binds).  BM = 256, three stages of 32 + 32 KB; the two
-//          accumulators hold the two row halves of one item, which halves the bytes the SM
-//          pulls from L2 per MMA.  Within a stage the MMAs of the first half are issued
+//          accumulators hold the two row halves of one item, which takes a third off the
+//          bytes the SM pulls from L2 per MMA.  Within a stage the MMAs of the first half are issued
 //          first, so its read-out overlaps the last MMAs of the second half, and the read-out
 //          of the second half the first MMAs of the next item.
 //
