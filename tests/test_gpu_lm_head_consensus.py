@@ -85,6 +85,9 @@ def rand_case(B, K, V, H, seed):
     (1, 1, 7, 8),            # the smallest everything
     (4, 32, 2048, 1024),     # exact tiles, 16 stages per item
     (1, 16, 4099, 4096),     # the hidden size of the 8B-class configurations
+    (64, 64, 1000, 128),     # 4096 rows: sixteen 256-row tiles
+    (2, 100, 777, 200),      # 200 rows (one 256-row tile, ragged), hidden 200 = 3 stages + 8 columns
+    (5, 26, 300, 64),        # 130 rows: two rows past the 128-row shape
 ])
 def test_fused_matches_oracle(B, K, V, H):
     hidden, lm_head = rand_case(B, K, V, H, seed=B * 1000 + K + V + H)
