@@ -308,6 +308,24 @@ class DeviceState:
         return self.res_host.numel() * 4 + self.out_host[0].numel() * self.out_host[0].element_size()
 
 
+def read_bandwidth_probe(dev, stream) -> float:
+    """Read-only streaming bandwidth of this GPU right now (GB/s): a second denominator for a
+    path that reads far more than it writes (the measured peak is a copy: read + write)."""
+    n = 1 << 30
+    x = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    x.fill_(1.0)
+    best = 0.0
+    for _ in range(6):
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        y = x.sum(dtype=torch.float32)
+        e1.record(stream)
+        stream.synchronize()
+        best = max(best, 2.0 * n / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    del x, y
+    return best
+
+
 def capture(fn, stream):
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g, stream=stream):
@@ -394,6 +412,8 @@ def run_gpu(args):
 
         total_ms = evs[0][0].elapsed_time(evs[-1][4])
         phase_ms = [statistics.mean(e[i].elapsed_time(e[i + 1]) for e in evs) for i in range(4)]
+        per_step = [e[0].elapsed_time(e[4]) for e in evs]
+        read_probe = read_bandwidth_probe(dev, stream)
         n_commit = st.n_commit.cpu()
         status = B.orthrus_read_status(st.ws, stream)
 
@@ -447,7 +467,14 @@ def run_gpu(args):
                    "multi_gpu": "replicas only"},
         "pct_of_hbm_peak": {"of_measured_%.0f" % peak if peak_kind == "measured" else
                             "of_fallback_%.0f" % peak: round(100 * kv_gbs / world / peak, 2),
-                            "of_nominal_8000": round(100 * kv_gbs / world / NOMINAL_HBM_GBS, 2)},
+                            "of_nominal_8000": round(100 * kv_gbs / world / NOMINAL_HBM_GBS, 2),
+                            "of_read_probe_%.0f" % read_probe: round(100 * kv_gbs / world / read_probe, 2)},
+        "read_probe": {"gbs": round(read_probe, 1),
+                       "how": "library reduction (torch.sum) over 2 GiB of bf16, best of 5, CUDA events"},
+        "kv_gbs_per_view": {"diffusion": round(call_bytes * layers / (phase_ms[0] * 1e-3) / 1e9, 2),
+                            "ar_verify": round(call_bytes * layers / (phase_ms[1] * 1e-3) / 1e9, 2)},
+        "ms_per_step_median": round(statistics.median(per_step), 5),
+        "ms_per_step_min": round(min(per_step), 5),
         "verified_tokens_per_s": round(world * tokens / (ms_per_step * 1e-3), 1),
         "verified_tokens_per_step": tokens,
         "tokens_per_forward_pass": round(tokens / wl.batch / 2.0, 4),
