@@ -498,6 +498,9 @@ def run_gpu(args):
         with torch.cuda.stream(stream):
             out["lm_head_consensus"] = lm_head_measure(B, wl, args.lm_head, dev, stream,
                                                        max(3, min(args.steps, 50)), local)
+    if args.decoder_cycles > 0:
+        with torch.cuda.stream(stream):
+            out["decoder_loop"] = decoder_loop_measure(B, dev, stream, args.decoder_cycles)
     if rank == 0:
         if not args.no_cpu_baseline and world == 1:
             out["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_budget, gpu_state=st)
@@ -597,6 +600,120 @@ def lm_head_measure(B, wl, hidden_dim, dev, stream, steps, gpu_index=0):
                           "tflops": round(flops / (ms_long * 1e-3) / 1e12, 2),
                           "lm_head_gbs": round(nbytes / (ms_long * 1e-3) / 1e9, 1), "clocks": long_clocks},
             "roofline": roof}
+
+
+def decoder_loop_measure(B, dev, stream, cycles):
+    """Whole generation cycles of a random-initialised decoder with the shapes of the
+    end-to-end configuration (12 layers, hidden 2048, 16/4 heads of 128, FFN 5632, vocabulary
+    32000, 8 sequences, prompts of 2048 tokens, block 16; about 1.2 GB of bf16 weights per
+    forward pass).  Everything off the hot path is plain torch (library GEMMs); both attention
+    passes, the LM-head-fused consensus and the commit go through the C ABI.  Drafts are forced
+    to agree with the AR view's precomputed greedy trajectory at a rate of 0.65 per position
+    (the diffusion view of a random-initialised model proposes nothing useful; once a sequence
+    leaves the precomputed trajectory at a near-tie its drafts stop agreeing), the diffusion
+    pass still runs in full.  One cycle is captured in a CUDA graph and replayed; the library's
+    share is the replay time of a second graph holding only that cycle's library calls."""
+    from paper_2605_12825_b200.decoder_harness import Decoder
+    layers, hidden, n_q, n_kv, d, ffn, vocab = 12, 2048, 16, 4, 128, 5632, 32000
+    Bt, T, K, rate = 8, 2048, 16, 0.65
+    n_traj = (cycles + 8) * K
+    cap = T + n_traj + 2 * K + 8
+    g = torch.Generator().manual_seed(W.sub_seed(W.BASE_SEED, "cfg5_loop", 0, "prompt"))
+    prompt = torch.randint(0, vocab, (Bt, T), generator=g).to(dev)
+    dec = Decoder(B, layers, hidden, n_q, n_kv, d, ffn, vocab, torch.bfloat16, Bt, cap, K, seed=5,
+                  flags=B.LAYER_CACHE_QUIESCENT)
+    i32 = dict(dtype=torch.int32, device=dev)
+    head = dec.lm_head_rows()
+    anchor0 = dec.prefill(prompt)
+    len0 = dec.cache_len.clone()
+    # the AR view's greedy trajectory (width-1 decoding), then rewind the cache length
+    outs1 = [torch.zeros(Bt, **i32), torch.zeros(Bt, 1, **i32), torch.zeros(Bt, 1, **i32), torch.zeros(Bt, **i32)]
+    ws1 = B.new_workspace(B.orthrus_lm_head_consensus_workspace_bytes(Bt, 1, vocab), device=dev)
+    zero1 = torch.zeros(Bt, 1, **i32)
+    traj, anchor = [], anchor0
+    for _ in range(n_traj):
+        _, ks, vs, hn = dec.forward_block(anchor.view(Bt, 1), "ar", 1, return_hidden=True, want_logits=False)
+        B.orthrus_lm_head_consensus(hn, head, zero1, *outs1, ws1)
+        dec.commit(ks, vs, outs1[0], 1)
+        anchor = outs1[3].clone()
+        traj.append(anchor)
+    traj = torch.stack(traj, 1)                                   # [B][n_traj]
+    dec.cache_len.copy_(len0)
+    wsK = B.new_workspace(B.orthrus_lm_head_consensus_workspace_bytes(Bt, K, vocab), device=dev)
+    done = torch.zeros(Bt, dtype=torch.int64, device=dev)
+    tokens = torch.zeros((), dtype=torch.int64, device=dev)
+    anchor = anchor0.clone()
+    ar = torch.arange(K, device=dev)
+
+    def cycle(record=None):
+        coin = torch.rand(Bt, K, device=dev) < rate
+        rnd = torch.randint(0, vocab, (Bt, K), device=dev, dtype=torch.int32)
+        idx = (done.view(Bt, 1) + ar).clamp(max=n_traj - 1)
+        draft = torch.where(coin, torch.gather(traj, 1, idx), rnd).to(torch.int32)
+        blk = torch.full((Bt, K), vocab, **i32)
+        blk[:, 0] = anchor
+        dec.forward_block(blk, "diff", K, want_logits=False, record=record)
+        ar_in = torch.cat([anchor.view(Bt, 1), draft[:, :K - 1]], dim=1)
+        _, ks, vs, hn = dec.forward_block(ar_in, "ar", K, return_hidden=True, want_logits=False, record=record)
+        tail = (lambda: (B.orthrus_lm_head_consensus(hn, head, draft, dec.n_commit, dec.committed, dec.ar_argmax,
+                                                     dec.next_anchor, wsK),
+                         dec.commit(ks, vs, dec.n_commit, K)))
+        tail()
+        if record is not None:
+            record.append(tail)
+        done.add_(dec.n_commit.long())
+        tokens.add_(dec.n_commit.sum())
+        anchor.copy_(dec.next_anchor)
+
+    for _ in range(3):
+        cycle()
+    stream.synchronize()
+    n0 = B.orthrus_launch_count()
+    g_cycle = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_cycle, stream=stream):
+        cycle()
+    launches = B.orthrus_launch_count() - n0
+    calls = []
+    cycle(calls)                                                  # eager, records the library calls
+    stream.synchronize()
+    len_mid = dec.cache_len.clone()
+    g_lib = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_lib, stream=stream):
+        for f in calls:
+            f()
+    dec.cache_len.copy_(len_mid)
+
+    def timed(graph, n, rewind):
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            graph.replay()
+            if rewind:
+                dec.cache_len.copy_(len_mid)
+        e1.record(stream)
+        stream.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    timed(g_lib, 3, True)
+    lib_ms = timed(g_lib, cycles, True)
+    timed(g_cycle, 2, False)
+    tokens.zero_()
+    ms = timed(g_cycle, cycles, False)
+    n_tok = int(tokens)
+    status = B.orthrus_read_status(dec.ws, stream) | B.orthrus_read_status(wsK, stream)
+    if status != 0:
+        raise SystemExit(f"bench.py: device status word {status} after the decoder loop")
+    return {"cycles": cycles, "ms_per_cycle": round(ms, 4),
+            "verified_tokens_per_s": round(n_tok / cycles / (ms * 1e-3), 1),
+            "verified_tokens_per_cycle": round(n_tok / cycles, 3),
+            "tokens_per_forward_pass": round(n_tok / cycles / Bt / 2.0, 4),
+            "in_library_ms_per_cycle": round(lib_ms, 4),
+            "in_library_share": round(lib_ms / ms, 4),
+            "library_launches_per_cycle": launches,
+            "model": {"layers": layers, "hidden": hidden, "q_heads": n_q, "kv_heads": n_kv, "head_dim": d,
+                      "ffn": ffn, "vocab": vocab, "batch": Bt, "prompt": T, "block": K,
+                      "forced_draft_agreement": rate, "weights": "random-initialised bf16",
+                      "off_path": "torch (library GEMMs), the whole cycle replayed from one CUDA graph"}}
 
 
 # ----------------------------------------------------------------------------- oracle arm
@@ -729,6 +846,9 @@ def main():
                     help="override the block width K (the block-size sweep of Section 5)")
     ap.add_argument("--lm-head", type=int, default=0, metavar="HIDDEN",
                     help="also time the fused LM-head consensus at this hidden size (extra key)")
+    ap.add_argument("--decoder-cycles", type=int, default=0, metavar="N",
+                    help="also time N whole generation cycles of the random-initialised decoder of the "
+                         "end-to-end configuration (extra key)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-early-prefetch", action="store_true",
                     help="do not set ORTHRUS_LAYER_CACHE_QUIESCENT on the layers")
