@@ -64,7 +64,7 @@ class Workload:
         return dataclasses.replace(self, **kw)
 
 
-# The five configurations of the build's baseline description, in order.
+# The five synthetic configurations, smallest first (the second is the one the headline metric is quoted on).
 CONFIGS: Dict[str, Workload] = {
     "cfg1_tiny": Workload("cfg1_tiny", 1, 8, 2, 64, 8, 1000, 512, 512,
                           layers=1, value_std=1.0 / 8, logit_std=1.0,
