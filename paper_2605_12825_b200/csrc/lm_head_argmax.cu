@@ -257,12 +257,13 @@ lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const in
 // Each CTA reads its 128 result rows out of its own TMEM.
 //
 // Barriers (same offsets in both CTAs): both producers' loads complete on the leader's FULL
-// barrier; the leader's MMA warp commits to the EMPTY and TFULL barriers of both CTAs with
-// one multicast commit; the read-out warps of both CTAs arrive on the leader's TEMPTY barrier.
-// The loads name no multicast.
+// barrier; the leader's MMA warp commits to the EMPTY and TFULL barriers of both CTAs (one
+// commit each); the read-out warps of both CTAs arrive on the leader's TEMPTY barrier.  No
+// load or commit is a cluster broadcast.
 //
-// Measured on the serving shape (1024 x 128256 x 4096) it equals the one-SM 256-row shape
-// (735 against 732 us): both run at the power cap, so the one-SM shape stays the default.
+// Measured on the serving shape (1024 x 128256 x 4096): 769 us against 750 us for the one-SM
+// 256-row shape on the same box (735 against 732 us with a single broadcast commit per stage
+// in a scratch build): both run at the power cap, so the one-SM shape stays the default.
 namespace pair {
 constexpr int NSTAGE = 3;
 constexpr int NTHREADS = 192;
@@ -298,10 +299,11 @@ __device__ inline void tma_load_2d_pair(uint32_t dst, const CUtensorMap *tm, int
                  " [%0], [%1, {%2, %3}], [%4], %5;"
                  ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(bar_cluster), "l"(policy) : "memory");
 }
-// the same arrival on the barrier at this offset in both CTAs of the pair
+// the same arrival on the barrier at this offset in both CTAs of the pair: one commit per CTA,
+// the peer's barrier addressed through the cluster window
 __device__ inline void umma_commit_both(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"((unsigned short)3) : "memory");
+    umma_commit_pair(bar);
+    umma_commit_pair(map_to_rank(bar, 1));
 }
 __device__ inline void mbar_arrive_cluster(uint32_t bar_cluster) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
