@@ -159,6 +159,9 @@ __global__ void __launch_bounds__(256) consensus_finalize_wide_kernel(
 {
     extern __shared__ int g[];
     const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // launched early (programmatic dependent launch): the pairs are complete once the kernel
+    // that writes them has finished
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int i = warp; i < K; i += 8) {
         const ArgPart *pp = parts + ((long long)b * K + i) * n_seg;
         float bv = -INFINITY;
@@ -198,10 +201,22 @@ cudaError_t launch_consensus_finalize_wide(const ArgPart *parts, int n_seg, cons
                                            int K, int32_t *n_commit, int32_t *committed,
                                            int32_t *ar_argmax, int32_t *next_anchor, cudaStream_t st)
 {
-    consensus_finalize_wide_kernel<<<B, 256, K * sizeof(int), st>>>(parts, n_seg, draft, K, n_commit,
-                                                                     committed, ar_argmax, next_anchor);
+    // programmatic dependent launch: the CTAs are placed while the producer of `parts` is still
+    // running and wait for it on the device
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(B);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = K * sizeof(int);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, consensus_finalize_wide_kernel, parts, n_seg, draft, K, n_commit,
+                                       committed, ar_argmax, next_anchor);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 int consensus_segments(int B, int K, int V)

@@ -137,6 +137,7 @@ lm_head_argmax_kernel(const __grid_constant__ HeadMaps tm, const int R, const in
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    griddep_launch();                         // the finalize kernel may be placed now; it waits for this grid
 
     // accumulator and its use count for row half `a` of this CTA's item number `li`
     auto acc_of = [](int li, int a) { return MT == 1 ? (li & 1) : a; };
@@ -348,6 +349,7 @@ lm_head_argmax_pair_kernel(const __grid_constant__ HeadMaps tm, const int R, con
     cluster_sync_all();                       // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    griddep_launch();                         // the finalize kernel may be placed now; it waits for this grid
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer (both CTAs)
