@@ -613,7 +613,7 @@ def decoder_loop_measure(B, dev, stream, cycles):
     leaves the precomputed trajectory at a near-tie its drafts stop agreeing), the diffusion
     pass still runs in full.  One cycle is captured in a CUDA graph and replayed; the library's
     share is the replay time of a second graph holding only that cycle's library calls."""
-    from paper_2605_12825_b200.decoder_harness import Decoder
+    from harness.decoder import Decoder
     layers, hidden, n_q, n_kv, d, ffn, vocab = 12, 2048, 16, 4, 128, 5632, 32000
     Bt, T, K, rate = 8, 2048, 16, 0.65
     n_traj = (cycles + 8) * K

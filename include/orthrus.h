@@ -50,12 +50,15 @@ typedef enum {
     ORTHRUS_ERR_UNSUPPORTED = 2,  /* shape or dtype outside the supported set     */
     ORTHRUS_ERR_CAPACITY = 3,     /* max_len_hint + block exceeds capacity        */
     ORTHRUS_ERR_WORKSPACE = 4,    /* workspace smaller than *_workspace_bytes()   */
-    ORTHRUS_ERR_CUDA = 5          /* a CUDA runtime call failed                   */
+    ORTHRUS_ERR_CUDA = 5,         /* a CUDA runtime call failed                   */
+    ORTHRUS_ERR_TIMEOUT = 6       /* orthrus_read_status only: the status word has
+                                     ORTHRUS_DEV_WAIT_TIMEOUT set                  */
 } orthrus_status_t;
 
 /* bits of the device status word (first int32 of the workspace) */
 enum {
-    ORTHRUS_DEV_BAD_CACHE_LEN = 1,   /* cache_len[b] outside [0, capacity-K]: clamped      */
+    ORTHRUS_DEV_BAD_CACHE_LEN = 1,   /* cache_len[b] outside [0, capacity-K], or above a
+                                        max_len_hint the launch was sized for: clamped      */
     ORTHRUS_DEV_APPEND_OVERFLOW = 2, /* cache_len[b]+n_commit[b] > capacity, or n_commit[b]
                                         outside [0,K]: that sequence was not appended       */
     ORTHRUS_DEV_WAIT_TIMEOUT = 4     /* a bounded hardware wait expired; outputs undefined  */
@@ -76,7 +79,9 @@ typedef struct {
     void *v_cache;          /* device [B][Hkv][capacity][d]                         */
     int32_t *cache_len;     /* device [B]: prefix length P_b, 0 <= P_b <= cap - K   */
     int32_t max_len_hint;   /* host upper bound on every P_b; sizes the split-KV
-                               grid.  0 means capacity - block                      */
+                               grid.  0 means capacity - block.  A P_b above the
+                               hint may be clamped to what the grid covers (then
+                               ORTHRUS_DEV_BAD_CACHE_LEN is raised)                 */
     float softmax_scale;    /* 0 selects 1/sqrt(head_dim), the scale of Eq. 4       */
     uint32_t flags;         /* OR of ORTHRUS_LAYER_* bits, 0 for none               */
 } orthrus_layer_t;
@@ -105,7 +110,8 @@ enum {
  * Bytes of workspace the two attention calls (and orthrus_kv_append) need for
  * this layer shape: a 256-byte header holding the status word, followed by the
  * split-KV partial results (written and read back inside one call; they are meant
- * to stay in L2).  A workspace serves one stream at a time: calls on the same stream
+ * to stay in L2).  Sizes depend on the device (its SM count shapes the split plan):
+ * ask with the device current that will run the calls.  A workspace serves one stream at a time: calls on the same stream
  * may share it, calls that can overlap on the GPU (different streams) need their own.
  * Returns 0 for an invalid descriptor.
  */
@@ -275,6 +281,9 @@ orthrus_status_t orthrus_kv_append_layers(const orthrus_layer_t *layers, int32_t
 /*
  * Copies the device status word to *host_status and waits for the stream (the
  * only call here that synchronises).  0 means no device-side problem so far.
+ * Returns ORTHRUS_ERR_TIMEOUT (with *host_status filled in) if the word has
+ * ORTHRUS_DEV_WAIT_TIMEOUT set: the outputs of the calls since the word was last
+ * cleared are undefined; the other bits are advisory and return ORTHRUS_OK.
  */
 orthrus_status_t orthrus_read_status(const void *workspace, void *stream, int32_t *host_status);
 

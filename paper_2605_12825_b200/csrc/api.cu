@@ -42,6 +42,29 @@ static int env_int(const char *name, int dflt)
     return v > 0 ? v : dflt;
 }
 
+}  // namespace orthrus
+
+int orthrus::num_sms()
+{
+    constexpr int kMaxDevices = 64;
+    static std::atomic<int> cached[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return kDefaultSMs;
+    }
+    int n = cached[dev].load(std::memory_order_relaxed);
+    if (n > 0) return n;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+        (void)cudaGetLastError();
+        return kDefaultSMs;
+    }
+    cached[dev].store(n, std::memory_order_relaxed);
+    return n;
+}
+
+namespace orthrus {
+
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 static orthrus_status_t check_layer(const orthrus_layer_t *L)
@@ -79,6 +102,15 @@ static bool tc_shape(const orthrus_layer_t *L)
            tc_row_tiles(L->n_q_heads / L->n_kv_heads, L->block) > 0;
 }
 
+// The tcgen05 path as a whole: the shape, the row count a 2-D tensor map can index and a
+// driver that offers the tensor-map encoder.  Anything else plans and launches on mma / SIMT.
+static bool tc_usable(const orthrus_layer_t *L)
+{
+    if (!tc_shape(L)) return false;
+    const unsigned long long rows = (unsigned long long)L->batch * L->n_kv_heads * (unsigned long long)L->capacity;
+    return rows < 0x7fffffffull && tc_driver_ok();
+}
+
 static Plan make_plan(const orthrus_layer_t *L, bool tc)
 {
     const int max_len = max_len_of(L);
@@ -90,7 +122,7 @@ static Plan make_plan(const orthrus_layer_t *L, bool tc)
         // to fill every slot once; sequences of unequal length are handed out longest first.
         const int tn = tc_tile_positions();
         const int units = L->batch * L->n_kv_heads * tc_row_tiles(L->n_q_heads / L->n_kv_heads, L->block);
-        const int slots = tc_ctas_per_sm() * kNumSMs;
+        const int slots = tc_ctas_per_sm() * num_sms();
         const int tiles = max_len > 0 ? (max_len + tn - 1) / tn : 1;
         int S = 1;
         if (forced > 0) {
@@ -115,7 +147,7 @@ static Plan make_plan(const orthrus_layer_t *L, bool tc)
     const int granule = 128;
     const int units = L->batch * L->n_kv_heads;
     const int tiles = max_len > 0 ? (max_len + granule - 1) / granule : 1;
-    const int target = env_int("ORTHRUS_TARGET_CTAS", 2 * kNumSMs);
+    const int target = env_int("ORTHRUS_TARGET_CTAS", 2 * num_sms());
     const int min_chunk_tiles = env_int("ORTHRUS_MIN_CHUNK_TILES", 2);
     int splits = (target + units - 1) / units;
     if (forced > 0) splits = forced;
@@ -160,7 +192,7 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
         (reinterpret_cast<uintptr_t>(L->cache_len) & 3))
         return ORTHRUS_ERR_INVALID_ARG;
     const int want = current_path();
-    const bool tc = (want == PATH_AUTO || want == PATH_TCGEN05) && tc_shape(L);
+    const bool tc = (want == PATH_AUTO || want == PATH_TCGEN05) && tc_usable(L);
     const Plan pl = make_plan(L, tc);
     size_t ml_off = 0;
     const size_t need = kHeaderBytes + partial_bytes(L, pl, &ml_off, tc);
@@ -182,14 +214,12 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     cudaError_t e;
     bool merge_kernel = pl.n_splits > 1;
-    if (tc && tc_path_supports(p, L->dtype)) {
+    if (tc) {
         t_last_path = "tcgen05";
         int flags = (int)(L->flags & (ORTHRUS_LAYER_CACHE_QUIESCENT | ORTHRUS_LAYER_NO_EARLY_LAUNCH));
         if (env_int("ORTHRUS_NO_EARLY_LAUNCH", 0)) flags |= ORTHRUS_LAYER_NO_EARLY_LAUNCH;
         e = launch_attend_tc(p, flags, cs);
         merge_kernel = false;
-    } else if (tc) {
-        return ORTHRUS_ERR_CUDA;            // the driver offers no tensor-map encoder
     } else if (want != PATH_SIMT && mma_path_supports(p, L->dtype)) {
         t_last_path = "mma";
         e = launch_attend_mma(p, cs);
@@ -216,7 +246,7 @@ size_t orthrus_attend_workspace_bytes(const orthrus_layer_t *layer)
     if (check_layer(layer) != ORTHRUS_OK) return 0;
     // enough for whichever kernel path a later call resolves to
     size_t need = partial_bytes(layer, make_plan(layer, false), nullptr, false);
-    if (tc_shape(layer)) {
+    if (tc_usable(layer)) {
         const size_t n2 = partial_bytes(layer, make_plan(layer, true), nullptr, true);
         if (n2 > need) need = n2;
     }
@@ -432,7 +462,8 @@ orthrus_status_t orthrus_read_status(const void *workspace, void *stream, int32_
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(host_status, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, cs) != cudaSuccess)
         return ORTHRUS_ERR_CUDA;
-    return cudaStreamSynchronize(cs) == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+    if (cudaStreamSynchronize(cs) != cudaSuccess) return ORTHRUS_ERR_CUDA;
+    return (*host_status & ORTHRUS_DEV_WAIT_TIMEOUT) ? ORTHRUS_ERR_TIMEOUT : ORTHRUS_OK;
 }
 
 orthrus_status_t orthrus_set_path(const char *name)
@@ -456,10 +487,11 @@ const char *orthrus_status_string(orthrus_status_t status)
     case ORTHRUS_ERR_CAPACITY: return "block does not fit in the cache capacity";
     case ORTHRUS_ERR_WORKSPACE: return "workspace too small";
     case ORTHRUS_ERR_CUDA: return "CUDA runtime error";
+    case ORTHRUS_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
     }
     return "unknown status";
 }
 
-int32_t orthrus_version(void) { return 100; }
+int32_t orthrus_version(void) { return 200; }
 
 }  // extern "C"

@@ -782,14 +782,28 @@ int tc_row_tiles(int G, int K)
     return (K + kb - 1) / kb;
 }
 
-bool tc_path_supports(const AttnParams &p, int dtype)
-{
-    if (dtype != ORTHRUS_BF16 || p.d != HD || p.K > TN || p.G > MROWS) return false;
-    const unsigned long long rows = (unsigned long long)p.B * p.Hkv * p.capacity;
-    return rows < 0x7fffffffull && encode_fn() != nullptr;
-}
+bool tc_driver_ok() { return encode_fn() != nullptr; }
 
-int tc_ctas_per_sm() { return 2; }
+// CTAs of this kernel one SM of the current device keeps resident (2 on a B200: shared memory
+// binds); asked once per device, 2 assumed where there is no device to ask.
+int tc_ctas_per_sm()
+{
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static int cached[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { (void)cudaGetLastError(); return 2; }
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[dev]) return cached[dev];
+    int n = 0;
+    if (cudaFuncSetAttribute(attend_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attend_tc_kernel<1>, NTHREADS, SMEM_BYTES) != cudaSuccess || n < 1) {
+        (void)cudaGetLastError();
+        return 2;
+    }
+    cached[dev] = n;
+    return n;
+}
 
 // Largest cluster size (a power of two up to 16) the current device can co-schedule for this
 // kernel; 16 on a full B200.  Without a device (or if the query fails) 16 is assumed and a

@@ -16,10 +16,11 @@ __global__ void __launch_bounds__(256) combine_kernel(AttnParams p)
     const int R = blockIdx.y * 8 + warp;
     if (R >= p.M) return;
     const int b = unit / p.Hkv, h = unit % p.Hkv;
+    // the same clamp as the kernels that wrote the partial rows (they raised the status bit)
     int P = p.cache_len[b];
-    const long long hi = p.capacity - p.K;
+    const long long hi = max_served_len(p);
     P = P < 0 ? 0 : (P > hi ? (int)hi : P);
-    const int ns = last_split(P, p.chunk) + 1;
+    const int ns = min(last_split(P, p.chunk) + 1, p.n_splits);
     const long long row0 = ((long long)unit * p.n_splits) * p.M + R;
 
     float mx = -INFINITY;

@@ -10,7 +10,11 @@ namespace orthrus {
 
 constexpr int kHeaderBytes = 256;       // workspace header; int32 status word at offset 0
 constexpr int kMaxSplits = 64;
-constexpr int kNumSMs = 148;
+constexpr int kDefaultSMs = 148;      // a full B200; used only when no device can be asked
+
+// Streaming multiprocessors of the current device (asked once per device; kDefaultSMs when
+// there is no device, so that size queries still work on a host without a GPU).
+int num_sms();
 
 // Parameters common to every attention kernel.  Rows of one (sequence, KV head)
 // unit are ordered r = i * G + g  (block position i, head g within the group), so
@@ -38,9 +42,17 @@ __host__ __device__ inline int last_split(int P, int chunk) {
     return P <= 0 ? 0 : (P - 1) / chunk;
 }
 
+// Largest prefix length a launch can serve: the capacity left beside the block, and (split-KV
+// grids of the SIMT / mma paths, sized from max_len_hint) what the planned splits cover.
+__host__ __device__ inline long long max_served_len(const AttnParams &p) {
+    const long long hi = p.capacity - p.K;
+    const long long planned = (long long)p.n_splits * p.chunk;
+    return planned < hi ? planned : hi;
+}
+
 __device__ inline int clamp_cache_len(const AttnParams &p, int b) {
     int P = p.cache_len[b];
-    long long hi = p.capacity - p.K;
+    const long long hi = max_served_len(p);
     if (P < 0 || P > hi) {
         if (p.status) atomicOr(p.status, ORTHRUS_DEV_BAD_CACHE_LEN);
         P = P < 0 ? 0 : (int)hi;
@@ -53,7 +65,7 @@ cudaError_t launch_attend_simt(const AttnParams &p, int dtype, cudaStream_t st);
 bool mma_path_supports(const AttnParams &p, int dtype);
 cudaError_t launch_attend_mma(const AttnParams &p, cudaStream_t st);
 int mma_tile_positions();
-bool tc_path_supports(const AttnParams &p, int dtype);
+bool tc_driver_ok();                    // the driver offers cuTensorMapEncodeTiled
 cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st);   // n_splits = cluster size
 int tc_row_tiles(int G, int K);          // 128-row query tiles per unit (0: group too wide)
 int tc_ctas_per_sm();

@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(256) argmax_partial_kernel(const T *logits, in
         if ((int)threadIdx.x < head) {
             const int i = start + threadIdx.x;
             const float x = Vec<T>::scalar(rowp + i);
-            if (better(x, i, bv, bi)) { bv = x; bi = i; }
+            if (x > bv) { bv = x; bi = i; }      // strict, like the body: -inf and NaN never replace the sentinel
         }
         const uint4 *vp = reinterpret_cast<const uint4 *>(rowp + body0);
         int v = threadIdx.x;
@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(256) argmax_partial_kernel(const T *logits, in
         if ((int)threadIdx.x < end - tail0) {
             const int i = tail0 + threadIdx.x;
             const float x = Vec<T>::scalar(rowp + i);
-            if (better(x, i, bv, bi)) { bv = x; bi = i; }
+            if (x > bv) { bv = x; bi = i; }      // strict, like the body: -inf and NaN never replace the sentinel
         }
     }
 #pragma unroll
@@ -222,7 +222,7 @@ cudaError_t launch_consensus_finalize_wide(const ArgPart *parts, int n_seg, cons
 int consensus_segments(int B, int K, int V)
 {
     const long long rows = (long long)B * K;
-    long long want = (4LL * kNumSMs + rows - 1) / rows;          // enough CTAs to fill the GPU
+    long long want = (4LL * num_sms() + rows - 1) / rows;          // enough CTAs to fill the GPU
     const long long max_by_len = (V + 2047) / 2048;              // at least 2048 logits each
     if (want > max_by_len) want = max_by_len;
     if (want < 1) want = 1;

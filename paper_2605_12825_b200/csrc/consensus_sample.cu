@@ -338,7 +338,7 @@ __global__ void __launch_bounds__(kThreads) sample_pick_kernel(const T *la, cons
 int sample_stat_segments(int B, int K, int V)
 {
     const long long rows = (long long)B * K;
-    long long want = (8LL * kNumSMs + rows - 1) / rows;           // more CTAs than fit at once, for balance
+    long long want = (8LL * num_sms() + rows - 1) / rows;           // more CTAs than fit at once, for balance
     const long long max_by_len = (V + 4095) / 4096;
     if (want > max_by_len) want = max_by_len;
     return (int)(want < 1 ? 1 : want);

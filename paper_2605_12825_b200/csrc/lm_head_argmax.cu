@@ -523,7 +523,7 @@ cudaError_t launch_shape(const HeadMaps &tm, int R, int V, int H, int bn, ArgPar
     }
     const int n_m = (R + S::BM - 1) / S::BM, n_n = (V + bn - 1) / bn, n_k = (H + BK - 1) / BK;
     const long long n_items = (long long)n_m * n_n;
-    const int grid = (int)(n_items < kNumSMs ? n_items : kNumSMs);
+    const int grid = (int)(n_items < num_sms() ? n_items : num_sms());
     lm_head_argmax_kernel<MT><<<grid, S::NTHREADS, S::SMEM_BYTES, st>>>(tm, R, V, n_k, n_m, n_n, bn, parts,
                                                                        status);
     count_launch();
@@ -548,7 +548,7 @@ int pair_clusters()
     if (cudaFuncSetAttribute(lm_head_argmax_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              pair::SMEM_BYTES) == cudaSuccess) {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(2 * kNumSMs, 1, 1);
+        cfg.gridDim = dim3(2 * num_sms(), 1, 1);
         cfg.blockDim = dim3(pair::NTHREADS);
         cfg.dynamicSmemBytes = pair::SMEM_BYTES;
         cudaLaunchAttribute attr[1];
@@ -558,7 +558,7 @@ int pair_clusters()
         if (cudaOccupancyMaxActiveClusters(&n, lm_head_argmax_pair_kernel, &cfg) != cudaSuccess) n = 0;
     }
     (void)cudaGetLastError();
-    if (n > kNumSMs / 2) n = kNumSMs / 2;
+    if (n > num_sms() / 2) n = num_sms() / 2;
     cached[dev] = n; known[dev] = true;
     return n;
 }
@@ -586,7 +586,7 @@ cudaError_t launch_pair(const HeadMaps &tm, int R, int V, int H, int bn, int clu
 static int tile_width(int R, int V, int pairs)
 {
     const int n_m = R > 128 ? (R + 255) / 256 : 1;
-    const int workers = pairs > 0 ? pairs : kNumSMs, step = pairs > 0 ? 32 : 16;
+    const int workers = pairs > 0 ? pairs : num_sms(), step = pairs > 0 ? 32 : 16;
     int best_bn = BN;
     long long best_cost = -1;
     for (int bn = BN; bn >= 128; bn -= step) {

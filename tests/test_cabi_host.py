@@ -33,8 +33,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_status_strings(lib):
-    s = {lib.lib().orthrus_status_string(c).decode() for c in range(6)}
-    assert len(s) == 6
+    s = {lib.lib().orthrus_status_string(c).decode() for c in range(7)}
+    assert len(s) == 7
 
 
 def _layer(lib, **kw):

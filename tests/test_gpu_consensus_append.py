@@ -59,6 +59,22 @@ def test_consensus_ties_and_special_values():
     assert n.tolist() == [4, 4]
 
 
+@pytest.mark.parametrize("V,dtype", [(1001, torch.float32), (4099, torch.bfloat16), (7, torch.bfloat16)])
+def test_consensus_rows_without_a_finite_value_on_ragged_vocabularies(V, dtype):
+    """Rows whose start or end is not 16-byte aligned have scalar head and tail elements:
+    a row of -inf (with or without a few NaN) must still resolve to token 0 there, and an
+    ordinary row next to it must not be disturbed by the odd alignment."""
+    lg = torch.randn(2, 3, V, generator=torch.Generator().manual_seed(4)).to(dtype)
+    lg[0, 0, :] = -float("inf")
+    lg[0, 1, :] = -float("inf"); lg[0, 1, 0] = float("nan"); lg[0, 1, V - 1] = float("nan")
+    lg[0, 2, :] = -float("inf"); lg[0, 2, V - 1] = -1e30                 # the only finite value, in the tail
+    lg[1, 0, :] = float("nan")
+    lg[1, 1, :] = -float("inf"); lg[1, 1, 1] = -float("inf"); lg[1, 1, 0] = -3.0   # head element wins
+    draft = torch.zeros(2, 3, dtype=torch.int32)
+    n, com, arg, nxt = check_consensus(lg, draft)
+    assert arg[0].tolist() == [0, 0, V - 1] and arg[1].tolist()[:2] == [0, 0]
+
+
 def test_consensus_all_agree_and_none_agree():
     wl = small_workload(4, 8, 1, 1, 32, 1, 1, V=2000)
     lg = W.logits(wl)

@@ -13,7 +13,7 @@ import pytest
 import torch
 
 import oracle
-from _decoder_harness import Decoder
+from harness.decoder import Decoder
 from _gpu_util import binding
 
 pytestmark = pytest.mark.gpu
