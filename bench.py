@@ -137,7 +137,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "100", "-i", str(self.index)],
+                 "-lms", "50", "-i", str(self.index)],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -169,9 +169,12 @@ class ClockSampler:
             for name, val in zip(names, f[4:8]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
+        bins = {}
+        for v in sm:
+            bins[str(int(v))] = bins.get(str(int(v)), 0) + 1
         return {"sm_mhz": statistics.median(sm) if sm else None,
                 "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "samples_by_sm_mhz": bins, "reasons": sorted(reasons)}
 
 
 # ----------------------------------------------------------------------------- GPU arm
@@ -180,7 +183,8 @@ class DeviceState:
     """All tensors of the workload on one GPU, one set per layer (layers are distinct
     buffers, so every timed read of a long-prefix workload misses L2)."""
 
-    def __init__(self, wl: W.Workload, layers: int, dev: torch.device, layer_flags: int = 0):
+    def __init__(self, wl: W.Workload, layers: int, dev: torch.device, layer_flags: int = 0,
+                 arenas: int = 1):
         from paper_2605_12825_b200 import binding as B
         self.B, self.wl, self.layers, self.dev = B, wl, layers, dev
         self.lens_host = W.prefix_lengths(wl)
@@ -207,14 +211,26 @@ class DeviceState:
             offs.append(total)
             total += (v.numel() * v.element_size() + 255) // 256 * 256
         self.step_host = torch.empty(total, dtype=torch.uint8).pin_memory()
-        self.step_dev = torch.empty(total, dtype=torch.uint8, device=dev)
+        # arena 0 serves the device-resident timing; with two arenas the end-to-end arm copies
+        # step s+1's inputs into one while step s computes on the other
+        self.step_devs = [torch.empty(total, dtype=torch.uint8, device=dev) for _ in range(arenas)]
+        self.step_dev = self.step_devs[0]
         self.step_bytes_h2d = total
-        views = {}
+        all_views = [dict() for _ in range(arenas)]
         for (l, k, v), off in zip(step_items, offs):
             nb = v.numel() * v.element_size()
             self.step_host[off:off + nb].view(v.dtype).view(v.shape).copy_(v)
-            views[(l, k)] = self.step_dev[off:off + nb].view(v.dtype).view(v.shape)
-        self.step_dev.copy_(self.step_host)
+            for a in range(arenas):
+                all_views[a][(l, k)] = self.step_devs[a][off:off + nb].view(v.dtype).view(v.shape)
+        for a in range(arenas):
+            self.step_devs[a].copy_(self.step_host)
+        views = all_views[0]
+        self.alt = []                      # per-step tensors of the other arenas: alt[a-1][l]
+        for a in range(1, arenas):
+            self.alt.append([{k: all_views[a][(l, k)] for k in host_layers[l] if "cache" not in k}
+                             for l in range(layers)])
+        self.alt_logits = [all_views[a][(-1, "logits")] for a in range(1, arenas)]
+        self.alt_draft = [all_views[a][(-1, "draft")] for a in range(1, arenas)]
         for l in range(layers):
             h = host_layers[l]
             t = {k: (v.to(dev) if "cache" in k else views[(l, k)]) for k, v in h.items()}
@@ -243,32 +259,41 @@ class DeviceState:
         self.ar_argmax = torch.zeros(Bn, K, **i32)
         self.next_anchor = torch.zeros(Bn, **i32)
         self.cws = B.new_workspace(B.orthrus_consensus_workspace_bytes(Bn, K, wl.vocab))
-        self.res_host = torch.zeros(Bn, dtype=torch.int32).pin_memory()
+        # what a caller needs back on the host every step: the consensus results (how many
+        # tokens, which, the next anchor); the attention outputs feed the next projection on
+        # the device and stay there, except the last layer's AR-view output, copied as a
+        # stand-in for whatever hidden state a caller may want to inspect
+        self.res_host = torch.zeros(Bn * (2 * K + 2), dtype=torch.int32).pin_memory()
         self.out_host = [torch.empty(t["q_diff"].shape, dtype=t["q_diff"].dtype).pin_memory()
                          for t in self.t[:1]]
 
+    def step_tensors(self, l, arena):
+        return self.t[l] if arena == 0 else self.alt[arena - 1][l]
+
     # the four phases of a step, each a sequence of C-ABI calls on the current stream
-    def phase_diffusion(self):
+    def phase_diffusion(self, arena=0):
         B = self.B
         for l in range(self.layers):
-            t = self.t[l]
+            t = self.step_tensors(l, arena)
             B.orthrus_diffusion_block_attend(self.layer0_first if l == 0 else self.layer[l], t["q_diff"],
                                              t["k_diff_blk"], t["v_diff_blk"], self.out_d[l], self.ws)
 
-    def phase_ar(self):
+    def phase_ar(self, arena=0):
         B = self.B
         for l in range(self.layers):
-            t = self.t[l]
+            t = self.step_tensors(l, arena)
             B.orthrus_ar_verify_attend(self.layer[l], t["q_ar"], t["k_ar_blk"], t["v_ar_blk"],
                                        self.out_a[l], self.ws)
 
-    def phase_consensus(self):
+    def phase_consensus(self, arena=0):
+        logits = self.logits if arena == 0 else self.alt_logits[arena - 1]
+        draft = self.draft if arena == 0 else self.alt_draft[arena - 1]
         if self.temperature > 0:
-            self.B.orthrus_consensus_sample(self.logits, self.diff_logits, self.draft, self.u_accept,
+            self.B.orthrus_consensus_sample(logits, self.diff_logits, draft, self.u_accept,
                                             self.u_resample, self.temperature, self.n_commit,
                                             self.committed, self.next_anchor, self.sws)
         else:
-            self.B.orthrus_consensus_accept(self.logits, self.draft, self.n_commit, self.committed,
+            self.B.orthrus_consensus_accept(logits, draft, self.n_commit, self.committed,
                                             self.ar_argmax, self.next_anchor, self.cws)
 
     def enable_sampling(self, temperature: float):
@@ -285,27 +310,39 @@ class DeviceState:
         self.sws = B.new_workspace(B.orthrus_consensus_sample_workspace_bytes(wl.batch, wl.block, wl.vocab))
         self.temperature = float(temperature)
 
-    def phase_commit(self):
+    def phase_commit(self, arena=0):
         # one launch commits the accepted rows of every layer; all layers share one length
         # array, which grows once
-        self.B.orthrus_kv_append_layers(self.layer, [t["k_ar_blk"] for t in self.t],
-                                        [t["v_ar_blk"] for t in self.t], self.n_commit, True, self.ws)
+        ts = [self.step_tensors(l, arena) for l in range(self.layers)]
+        self.B.orthrus_kv_append_layers(self.layer, [t["k_ar_blk"] for t in ts],
+                                        [t["v_ar_blk"] for t in ts], self.n_commit, True, self.ws)
         # the next step starts from the same prefix again (the appended bytes are identical
         # every step, so this rewinds the state exactly)
         self.cache_len.copy_(self.cache_len0)
 
-    def phases(self):
-        return [self.phase_diffusion, self.phase_ar, self.phase_consensus, self.phase_commit]
+    def phases(self, arena=0):
+        return [lambda: self.phase_diffusion(arena), lambda: self.phase_ar(arena),
+                lambda: self.phase_consensus(arena), lambda: self.phase_commit(arena)]
 
-    def h2d_inputs(self):
+    def h2d_inputs(self, arena=0):
         """End-to-end arm: this step's inputs come from pinned host memory, in one copy."""
-        self.step_dev.copy_(self.step_host, non_blocking=True)
+        self.step_devs[arena].copy_(self.step_host, non_blocking=True)
         return self.step_bytes_h2d
 
     def d2h_results(self):
-        self.res_host.copy_(self.n_commit, non_blocking=True)
+        Bn, K = self.wl.batch, self.wl.block
+        r = self.res_host
+        r[:Bn].copy_(self.n_commit, non_blocking=True)
+        r[Bn:2 * Bn].copy_(self.next_anchor, non_blocking=True)
+        r[2 * Bn:2 * Bn + Bn * K].view(Bn, K).copy_(self.committed, non_blocking=True)
+        r[2 * Bn + Bn * K:].view(Bn, K).copy_(self.ar_argmax, non_blocking=True)
         self.out_host[0].copy_(self.out_a[self.layers - 1], non_blocking=True)
-        return self.res_host.numel() * 4 + self.out_host[0].numel() * self.out_host[0].element_size()
+        return r.numel() * 4 + self.out_host[0].numel() * self.out_host[0].element_size()
+
+    def free(self):
+        for name in list(vars(self)):
+            if name not in ("wl", "layers", "lens_host"):
+                delattr(self, name)
 
 
 def read_bandwidth_probe(dev, stream) -> float:

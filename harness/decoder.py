@@ -42,6 +42,7 @@ class Decoder:
         self.cache_len = torch.zeros(batch, dtype=torch.int32, device=dev)
         self.flags = flags
         self.ws = None
+        self._ws_by_block = {}
         self.cws = binding.new_workspace(binding.orthrus_consensus_workspace_bytes(batch, block, vocab))
         i32 = dict(dtype=torch.int32, device=dev)
         self.n_commit = torch.zeros(batch, **i32)
@@ -99,20 +100,24 @@ class Decoder:
         return prompt[:, -1].to(torch.int32)
 
     # ------------------------------------------------------------------ one pass through the layers
-    def forward_block(self, tokens, view, block, return_hidden=False, want_logits=True, record=None):
+    def forward_block(self, tokens, view, block, return_hidden=False, want_logits=True, record=None,
+                      capture=None):
         """tokens [B][block] (id == vocab selects the mask embedding).  view 'diff' or 'ar'.
         Returns (logits [B][block][V], per-layer block K, per-layer block V), with
         return_hidden also the final-norm hidden states [B][block][H] the LM head is applied to.
         record: a list that receives one closure per library call (same arguments), so that a
-        caller can replay the library's share of the pass on its own."""
+        caller can replay the library's share of the pass on its own.
+        capture: a dict {layer index: None}; the entry of each listed layer is replaced by the
+        tensors of its attention call (q, k, v, out, cache_len; device clones), for parity checks."""
         b = self.b
         B = tokens.shape[0]
         h = self.emb[tokens.long()]
         pos = self.cache_len.long().unsqueeze(1) + torch.arange(block, device=h.device)
         layers = self.layer_objs(block)
-        if self.ws is None or self.ws_block != block:
-            self.ws = b.new_workspace(b.orthrus_attend_workspace_bytes(layers[0]))
-            self.ws_block = block
+        # one workspace per block width, kept for good: captured graphs hold its address
+        if block not in self._ws_by_block:
+            self._ws_by_block[block] = b.new_workspace(b.orthrus_attend_workspace_bytes(layers[0]))
+        self.ws = self._ws_by_block[block]
         sfx = "_d" if view == "diff" else ""
         ks, vs = [], []
         for l, lw in enumerate(self.layers):
@@ -122,8 +127,11 @@ class Decoder:
             v = (x @ lw["wv" + sfx]).view(B, block, self.Hkv, self.d).contiguous()
             out = torch.empty_like(q)
             fn = b.orthrus_diffusion_block_attend if view == "diff" else b.orthrus_ar_verify_attend
-            call = (lambda fn=fn, L=layers[l], q=q, k=k, v=v, out=out: fn(L, q, k, v, out, self.ws))
+            call = (lambda fn=fn, L=layers[l], q=q, k=k, v=v, out=out, ws=self.ws: fn(L, q, k, v, out, ws))
             call()
+            if capture is not None and l in capture:
+                capture[l] = dict(q=q.clone(), k=k.clone(), v=v.clone(), out=out.clone(),
+                                  cache_len=self.cache_len.clone())
             if record is not None:
                 record.append(call)
             h = h + out.view(B, block, self.Hq * self.d) @ lw["wo"]
@@ -143,3 +151,107 @@ class Decoder:
 
     def commit(self, ks, vs, n_commit, block):
         self.b.orthrus_kv_append_layers(self.layer_objs(block), ks, vs, n_commit, True, self.ws)
+
+    def status(self):
+        """OR of the device status words of every workspace this decoder has used."""
+        st = 0
+        for ws in self._ws_by_block.values():
+            st |= self.b.orthrus_read_status(ws)
+        return st
+
+
+class ForcedDraftLoop:
+    """The generation loop of Section 3.3 on a Decoder, with the diffusion view's drafts replaced by
+    forced ones so that acceptance is controlled (a random-initialised diffusion head proposes
+    nothing useful; its pass still runs in full).
+
+    Every cycle first looks ahead: `block` width-1 greedy steps of the AR view through the same
+    library calls give the tokens plain autoregressive decoding would emit next from the
+    current state; the cache length is then rewound (the rows the look-ahead wrote lie behind
+    it and are overwritten by the cycle's own commit).  Draft i is look-ahead token i with
+    probability `rate`, else a uniform token.  The look-ahead is also the reference of the
+    lossless check: the tokens a cycle commits must be its first n look-ahead tokens.  Because the
+    reference restarts from the loop's own state every cycle, a near-tie that block verification
+    and width-1 decoding round differently costs one mismatch and nothing after it."""
+
+    def __init__(self, dec, anchor, rate, seed=0, fused=True):
+        self.dec, self.rate, self.fused = dec, rate, fused
+        b, B, K, V = dec.b, dec.B, dec.K, dec.V
+        dev = anchor.device
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.anchor = anchor.clone()
+        self.anchor1 = anchor.clone()
+        self.draft = torch.zeros(B, K, **i32)
+        self.look = torch.zeros(B, K, **i32)
+        self.gaps = torch.zeros(B, K, dtype=torch.float32, device=dev)
+        self.done = torch.zeros(B, dtype=torch.int64, device=dev)
+        self.outs1 = [torch.zeros(B, **i32), torch.zeros(B, 1, **i32), torch.zeros(B, 1, **i32),
+                      torch.zeros(B, **i32)]
+        self.zero1 = torch.zeros(B, 1, **i32)
+        self.ws1 = b.new_workspace(b.orthrus_lm_head_consensus_workspace_bytes(B, 1, V), device=dev)
+        self.wsK = b.new_workspace(b.orthrus_lm_head_consensus_workspace_bytes(B, K, V), device=dev)
+        self.cws1 = b.new_workspace(b.orthrus_consensus_workspace_bytes(B, 1, V), device=dev)
+        self.gen = torch.Generator(device=dev)
+        self.gen.manual_seed(seed)
+        self.len_saved = dec.cache_len.clone()
+        self.logits = None            # AR logits of the last cycle (two-step consensus only)
+
+    # ---- width-1 reference steps
+    def k1_step(self, j, want_gap=False):
+        dec, b = self.dec, self.dec.b
+        logits, ks, vs, hn = dec.forward_block(self.anchor1.view(-1, 1), "ar", 1, return_hidden=True,
+                                               want_logits=want_gap or not self.fused)
+        if self.fused:
+            b.orthrus_lm_head_consensus(hn, dec.lm_head_rows(), self.zero1, *self.outs1, self.ws1)
+        else:
+            b.orthrus_consensus_accept(logits, self.zero1, *self.outs1, self.cws1)
+        if want_gap:
+            top2 = logits.float().topk(2, dim=-1).values[:, 0]
+            self.gaps[:, j] = top2[:, 0] - top2[:, 1]
+        dec.commit(ks, vs, self.outs1[0], 1)
+        self.anchor1.copy_(self.outs1[3])
+        self.look[:, j] = self.outs1[3]
+
+    def lookahead(self, want_gap=False):
+        dec = self.dec
+        self.len_saved.copy_(dec.cache_len)
+        self.anchor1.copy_(self.anchor)
+        for j in range(dec.K):
+            self.k1_step(j, want_gap)
+        dec.cache_len.copy_(self.len_saved)
+
+    def force_drafts(self):
+        B, K, V = self.dec.B, self.dec.K, self.dec.V
+        dev = self.draft.device
+        coin = torch.rand(B, K, device=dev, generator=self.gen) < self.rate
+        rnd = torch.randint(0, V, (B, K), device=dev, generator=self.gen, dtype=torch.int32)
+        self.draft.copy_(torch.where(coin, self.look, rnd))
+
+    # ---- one cycle: both passes, the consensus, the commit
+    def cycle(self, record=None, capture_diff=None, capture_ar=None):
+        dec, b = self.dec, self.dec.b
+        B, K, V = dec.B, dec.K, dec.V
+        blk = torch.full((B, K), V, dtype=torch.int32, device=self.draft.device)
+        blk[:, 0] = self.anchor
+        dec.forward_block(blk, "diff", K, want_logits=False, record=record, capture=capture_diff)
+        ar_in = torch.cat([self.anchor.view(B, 1), self.draft[:, :K - 1]], dim=1)
+        logits, ks, vs, hn = dec.forward_block(ar_in, "ar", K, return_hidden=True, want_logits=not self.fused,
+                                               record=record, capture=capture_ar)
+        self.logits = logits
+        if self.fused:
+            tail = (lambda: (b.orthrus_lm_head_consensus(hn, dec.lm_head_rows(), self.draft, dec.n_commit,
+                                                         dec.committed, dec.ar_argmax, dec.next_anchor, self.wsK),
+                             dec.commit(ks, vs, dec.n_commit, K)))
+        else:
+            tail = (lambda: (b.orthrus_consensus_accept(logits, self.draft, dec.n_commit, dec.committed,
+                                                        dec.ar_argmax, dec.next_anchor, dec.cws),
+                             dec.commit(ks, vs, dec.n_commit, K)))
+        tail()
+        if record is not None:
+            record.append(tail)
+        self.done.add_(dec.n_commit.long())
+        self.anchor.copy_(dec.next_anchor)
+
+    def status(self):
+        b = self.dec.b
+        return self.dec.status() | b.orthrus_read_status(self.ws1) | b.orthrus_read_status(self.wsK)

@@ -138,17 +138,19 @@ def test_length_above_the_hint_is_clamped_and_flagged_on_the_split_paths(path, d
     b.orthrus_set_path(path)
     try:
         nbytes = b.orthrus_attend_workspace_bytes(layer)
-        ws = Guarded((nbytes,), torch.uint8, pad=4096)
-        ws.buf.fill_(0x5A); ws.t.zero_()
+        pad = 4096
+        buf = torch.full((nbytes + 2 * pad,), 0x5A, dtype=torch.uint8, device="cuda")
+        ws = buf[pad:pad + nbytes]
+        ws.zero_()
         out = Guarded(tuple(t["q_ar"].shape), t["q_ar"].dtype)
-        b.orthrus_ar_verify_attend(layer, dev["q_ar"], dev["k_ar_blk"], dev["v_ar_blk"], out.t, ws.t)
+        b.orthrus_ar_verify_attend(layer, dev["q_ar"], dev["k_ar_blk"], dev["v_ar_blk"], out.t, ws)
         assert b.orthrus_last_path() == path
-        status = b.orthrus_read_status(ws.t)
+        status = b.orthrus_read_status(ws)
     finally:
         b.orthrus_set_path("auto")
     assert status & 1
     assert out.intact()
-    assert bool((ws.buf[:4096] == 0x5A).all()) and bool((ws.buf[4096 + nbytes:] == 0x5A).all())
+    assert bool((buf[:pad] == 0x5A).all()) and bool((buf[pad + nbytes:] == 0x5A).all())
     got = out.t.cpu()
     assert torch.isfinite(got.float()).all()
     # the clamped length is what the planned splits cover: at least the hint, a whole number of

@@ -1,0 +1,94 @@
+"""The end-to-end configuration at its stated size: a random-initialised 12-layer decoder
+(hidden 2048, 16 query / 4 KV heads of 128, SwiGLU FFN 5632, vocabulary 32000, bf16), 8
+prompts of 2048 tokens, then 256 generated tokens per sequence by repeated block-16 draft /
+verify / consensus / commit (Section 3.3), drafts forced to agree with greedy decoding at a
+rate of 0.65.
+
+Checked: every cycle's consensus equals the oracle's on the GPU's own logits, bit for bit; the
+cache length grows by n; the committed stream equals width-1 greedy decoding through the same
+library calls (restarted from the loop's state every cycle), except where the width-1 run's two
+largest logits are within a stated epsilon (block verification and width-1 decoding round
+differently in bf16; such events are counted); sampled attention rows of the first and the last
+layer, both views, against the oracle in the first cycle and in one more cycle after the last."""
+import pytest
+import torch
+
+import oracle
+from harness.decoder import Decoder, ForcedDraftLoop
+from _gpu_util import TOL, binding
+
+pytestmark = pytest.mark.gpu
+EPS_NEAR_TIE = 0.25
+
+
+def check_attention_rows(dec, captured, view, seed):
+    B, K, Hq = dec.B, dec.K, dec.Hq
+    g = torch.Generator().manual_seed(seed)
+    flat = torch.randperm(B * K * Hq, generator=g)[:48]
+    rows = torch.stack([flat // (K * Hq), (flat // Hq) % K, flat % Hq], dim=1).to(torch.int32)
+    atol, rtol = TOL[torch.bfloat16]
+    for l, c in captured.items():
+        assert c is not None, f"layer {l} was not captured"
+        ref = oracle.block_attend_rows(view, rows, c["q"].cpu(), c["k"].cpu(), c["v"].cpu(),
+                                       dec.k_cache[l].cpu(), dec.v_cache[l].cpu(), c["cache_len"].cpu())
+        got = c["out"].cpu().double()[rows[:, 0].long(), rows[:, 1].long(), rows[:, 2].long()]
+        err = float((got - ref).abs().max())
+        scale = float(ref.abs().max())
+        assert err <= atol and err <= rtol * scale, (l, view, err, scale)
+
+
+def test_generation_loop_of_the_end_to_end_configuration_at_full_size():
+    b = binding()
+    b.orthrus_set_path("auto")
+    layers, hidden, n_q, n_kv, d, ffn, vocab = 12, 2048, 16, 4, 128, 5632, 32000
+    B, T, K, n_new, rate = 8, 2048, 16, 256, 0.65
+    cap = T + n_new + 4 * K + 8
+    g = torch.Generator().manual_seed(12825)
+    prompt = torch.randint(0, vocab, (B, T), generator=g).cuda()
+    dec = Decoder(b, layers, hidden, n_q, n_kv, d, ffn, vocab, torch.bfloat16, B, cap, K, seed=5,
+                  flags=b.LAYER_CACHE_QUIESCENT)
+    anchor = dec.prefill(prompt)
+    loop = ForcedDraftLoop(dec, anchor, rate, seed=7, fused=False)
+
+    def one_cycle(capture):
+        loop.lookahead(want_gap=True)
+        loop.force_drafts()
+        len_before = dec.cache_len.cpu().clone()
+        cap_d = {0: None, layers - 1: None} if capture else None
+        cap_a = {0: None, layers - 1: None} if capture else None
+        loop.cycle(capture_diff=cap_d, capture_ar=cap_a)
+        assert b.orthrus_last_path() == "tcgen05"
+        rn, rcom, rarg, rnxt = oracle.consensus_accept(loop.logits.cpu(), loop.draft.cpu())
+        assert torch.equal(dec.n_commit.cpu(), rn) and torch.equal(dec.committed.cpu(), rcom)
+        assert torch.equal(dec.ar_argmax.cpu(), rarg) and torch.equal(dec.next_anchor.cpu(), rnxt)
+        assert int(rn.min()) >= 1 and int(rn.max()) <= K
+        assert torch.equal(dec.cache_len.cpu(), len_before + rn)
+        if capture:
+            check_attention_rows(dec, cap_d, oracle.VIEW_DIFFUSION, seed=int(len_before[0]))
+            check_attention_rows(dec, cap_a, oracle.VIEW_AR, seed=int(len_before[0]) + 1)
+        # lossless: the committed tokens are the width-1 greedy tokens, up to a near tie
+        look, gaps = loop.look.cpu(), loop.gaps.cpu()
+        ties = 0
+        for s in range(B):
+            for i in range(int(rn[s])):
+                if int(rcom[s, i]) != int(look[s, i]):
+                    assert float(gaps[s, i]) < EPS_NEAR_TIE, (s, i, int(rcom[s, i]), int(look[s, i]),
+                                                               float(gaps[s, i]))
+                    ties += 1
+                    break
+        return int(rn.sum()), ties
+
+    cycles, total, ties = 0, 0, 0
+    while int(loop.done.min()) < n_new:
+        n, t = one_cycle(capture=(cycles == 0))
+        total += n; ties += t; cycles += 1
+        assert cycles <= n_new, "the loop does not advance"
+    n, t = one_cycle(capture=True)           # one more cycle, on the longest cache
+    total += n; ties += t; cycles += 1
+    assert loop.status() == 0 and b.orthrus_read_status(dec.cws) == 0
+    mean_n = total / (cycles * B)
+    # E[n] = (1 - p^K) / (1 - p) = 2.85 for p = 0.65, K = 16; a near tie ends a cycle early
+    assert 2.0 < mean_n < 3.6, mean_n
+    assert ties <= total // 8, (ties, total)
+    print(f"config 5 at full size: {cycles} cycles, {total} tokens, mean n {mean_n:.3f}, "
+          f"{ties} near-tie resyncs")
