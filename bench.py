@@ -202,6 +202,8 @@ class DeviceState:
         host_layers = []
         for l in range(layers):
             h = W.attention_inputs(wl, layer=l)
+            if l == 0:
+                self.host0 = dict(h)              # kept for the oracle check of the timed outputs
             h.pop("cache_len")
             host_layers.append(h)
         step_items = [(l, k, v) for l, h in enumerate(host_layers) for k, v in h.items() if "cache" not in k]
@@ -370,6 +372,192 @@ def capture(fn, stream):
     return g
 
 
+class TimedWorkload:
+    """One workload on one GPU: device state, the captured phases and the timed region."""
+
+    def __init__(self, B, wl, layers, dev, stream, flags, arenas=1, temperature=0.0, no_graph=False):
+        self.B, self.wl, self.layers, self.dev, self.stream = B, wl, layers, dev, stream
+        self.st = DeviceState(wl, layers, dev, flags, arenas)
+        if temperature > 0:
+            self.st.enable_sampling(temperature)
+        st = self.st
+        with torch.cuda.stream(stream):
+            for a in range(arenas):
+                for _ in range(2):                  # eager warm-up (sets kernel attributes)
+                    for ph in st.phases(a):
+                        ph()
+            stream.synchronize()
+            n0 = B.orthrus_launch_count()
+            for ph in st.phases(0):
+                ph()
+            self.launches_per_step = B.orthrus_launch_count() - n0
+            stream.synchronize()
+            self.graphs = None
+            if not no_graph:
+                self.graphs = [[capture(ph, stream) for ph in st.phases(a)] for a in range(arenas)]
+
+    def step(self, events=None, arena=0):
+        stream = self.stream
+        phases = None if self.graphs is not None else self.st.phases(arena)
+        for i in range(4):
+            if events is not None:
+                events[i].record(stream)
+            if self.graphs is not None:
+                self.graphs[arena][i].replay()
+            else:
+                phases[i]()
+        if events is not None:
+            events[4].record(stream)
+
+    def run_timed(self, steps, warmup, min_region_s, gpu_index, dist=None):
+        """`steps` timed steps, each repeated `inner` times back to back so that the timed
+        region lasts at least `min_region_s`; events bracket every outer step and, in its
+        first repetition, every phase."""
+        stream = self.stream
+        with torch.cuda.stream(stream):
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            for _ in range(max(warmup, 3) - 1):
+                self.step()
+            e0.record(stream)
+            self.step()
+            e1.record(stream)
+            stream.synchronize()
+            est_ms = max(e0.elapsed_time(e1), 1e-3)
+            inner = max(1, int(math.ceil(min_region_s * 1e3 / (steps * est_ms))))
+            if dist is not None:
+                t = torch.tensor([inner], device=self.dev)
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                inner = int(t)
+                dist.barrier()
+            torch.cuda.synchronize()
+            sampler = ClockSampler(gpu_index)
+            sampler.start()
+            evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(steps)]
+            for s in range(steps):
+                self.step(evs[s])
+                for _ in range(inner - 1):
+                    self.step()
+                evs[s][5].record(stream)
+            stream.synchronize()
+            torch.cuda.synchronize()
+            clocks = sampler.stop()
+            if dist is not None:
+                dist.barrier()
+        total_ms = evs[0][0].elapsed_time(evs[-1][5])
+        return {"inner": inner, "ms_per_step": total_ms / (steps * inner),
+                "phase_ms": [statistics.mean(e[i].elapsed_time(e[i + 1]) for e in evs) for i in range(4)],
+                "per_step": [e[0].elapsed_time(e[5]) / inner for e in evs], "clocks": clocks}
+
+    def run_e2e(self, steps, overlap):
+        """The same step through host buffers: every step copies its inputs from pinned host
+        memory and its results back.  Serial: copy, compute, copy on one stream.  Overlapped:
+        two device arenas and a copy stream, so that step s+1's inputs cross the bus while step s
+        computes; a step still starts only when its own inputs have arrived."""
+        st, stream = self.st, self.stream
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        if not overlap:
+            with torch.cuda.stream(stream):
+                for _ in range(2):
+                    st.h2d_inputs(0); self.step(); st.d2h_results()
+                stream.synchronize()
+                e0.record(stream)
+                for _ in range(steps):
+                    h2d = st.h2d_inputs(0)
+                    self.step()
+                    d2h = st.d2h_results()
+                e1.record(stream)
+                stream.synchronize()
+            return e0.elapsed_time(e1) / steps, h2d, d2h
+        copy_stream = torch.cuda.Stream(device=self.dev)
+        arrived = [torch.cuda.Event() for _ in range(2)]
+        free = [torch.cuda.Event() for _ in range(2)]
+
+        def run(n):
+            for s in range(n):
+                a = s & 1
+                copy_stream.wait_event(free[a])            # the step that last used this arena is done
+                with torch.cuda.stream(copy_stream):
+                    h2d = st.h2d_inputs(a)
+                    arrived[a].record(copy_stream)
+                with torch.cuda.stream(stream):
+                    stream.wait_event(arrived[a])
+                    self.step(arena=a)
+                    d2h = st.d2h_results()
+                    free[a].record(stream)
+            return h2d, d2h
+
+        for a in range(2):
+            free[a].record(stream)
+        run(4)
+        stream.synchronize(); copy_stream.synchronize()
+        e0.record(stream)
+        h2d, d2h = run(steps)
+        e1.record(stream)
+        stream.synchronize(); copy_stream.synchronize()
+        return e0.elapsed_time(e1) / steps, h2d, d2h
+
+
+def check_against_oracle(wl, st, n_rows=48):
+    """A small sample of the timed step's outputs against the CPU oracle: `n_rows` attention rows
+    of both views of layer 0 under the parity tolerance, the consensus bit for bit."""
+    import oracle
+    oracle.build()
+    t = st.host0
+    g = torch.Generator().manual_seed(2)
+    Bn, K, Hq = wl.batch, wl.block, wl.n_q_heads
+    flat = torch.randperm(Bn * K * Hq, generator=g)[:n_rows]
+    rows = torch.stack([flat // (K * Hq), (flat // Hq) % K, flat % Hq], dim=1).to(torch.int32)
+    idx = (rows[:, 0].long(), rows[:, 1].long(), rows[:, 2].long())
+    worst = 0.0
+    for view, q, kb, vb, out in ((oracle.VIEW_DIFFUSION, "q_diff", "k_diff_blk", "v_diff_blk", st.out_d[0]),
+                                 (oracle.VIEW_AR, "q_ar", "k_ar_blk", "v_ar_blk", st.out_a[0])):
+        ref = oracle.block_attend_rows(view, rows, t[q], t[kb], t[vb], t["k_cache"], t["v_cache"], t["cache_len"])
+        err = float((out.cpu().double()[idx] - ref).abs().max())
+        scale = float(ref.abs().max())
+        if not (err <= 2e-2 and err <= 1e-2 * scale):
+            raise SystemExit(f"bench.py: {wl.name}: attention output of the timed step is off the oracle "
+                             f"(max-abs {err:.3e}, max|ref| {scale:.3e})")
+        worst = max(worst, err / scale)
+    cons = "not checked (sampled consensus)"
+    if st.temperature <= 0:
+        ref = oracle.consensus_accept(st.logits.cpu(), st.draft.cpu())
+        if not (torch.equal(st.n_commit.cpu(), ref[0]) and torch.equal(st.committed.cpu(), ref[1])):
+            raise SystemExit(f"bench.py: {wl.name}: consensus of the timed step differs from the oracle")
+        cons = "bit-exact"
+    return {"attention_rows": 2 * n_rows, "max_err_over_max_ref": round(worst, 5), "consensus": cons}
+
+
+def workload_entry(B, name, dev, stream, flags, steps, gpu_index, peak, min_region_s=0.25):
+    """Roofline and throughput of one more workload (all its layers), for the `workloads` key."""
+    wl = W.CONFIGS[name]
+    tw = TimedWorkload(B, wl, wl.layers, dev, stream, flags)
+    r = tw.run_timed(steps, 3, min_region_s, gpu_index)
+    st = tw.st
+    status = B.orthrus_read_status(st.ws, stream)
+    if status != 0:
+        raise SystemExit(f"bench.py: {name}: device status word {status} after the timed region")
+    call_bytes = attend_bytes(wl, st.lens_host)
+    attend_ms = (r["phase_ms"][0] + r["phase_ms"][1]) / (2 * wl.layers)
+    achieved = call_bytes / (attend_ms * 1e-3) / 1e9
+    tokens = int(st.n_commit.sum())
+    out = {"layers": wl.layers, "steps": steps, "inner_repeats": r["inner"],
+           "ms_per_step": round(r["ms_per_step"], 5),
+           "kv_gbs": round(call_bytes * 2 * wl.layers / (r["ms_per_step"] * 1e-3) / 1e9, 2),
+           "verified_tokens_per_s": round(tokens / (r["ms_per_step"] * 1e-3), 1),
+           "phase_ms": {"diffusion_attend": round(r["phase_ms"][0], 5), "ar_verify_attend": round(r["phase_ms"][1], 5),
+                        "consensus": round(r["phase_ms"][2], 5), "kv_commit": round(r["phase_ms"][3], 5)},
+           "roofline": {"bound": "hbm", "achieved": round(achieved, 2), "peak": peak, "unit": "GB/s",
+                        "frac": round(achieved / peak, 4), "algorithmic_bytes_per_launch": call_bytes,
+                        "avg_launch_us": round(attend_ms * 1e3, 3)},
+           "clocks": {k: r["clocks"].get(k) for k in ("sm_mhz", "samples", "reasons")},
+           "gpu_outputs_checked": check_against_oracle(wl, st)}
+    tw.graphs = None
+    st.free()
+    del tw, st
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_gpu(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -398,82 +586,33 @@ def run_gpu(args):
     flags = 0 if args.no_early_prefetch else B.LAYER_CACHE_QUIESCENT
     if args.no_early_launch:
         flags |= B.LAYER_NO_EARLY_LAUNCH
-    st = DeviceState(wl, layers, dev, flags)
-    if args.temperature > 0:
-        st.enable_sampling(args.temperature)
     stream = torch.cuda.Stream(device=dev)
-    phases = st.phases()
-
-    with torch.cuda.stream(stream):
-        for _ in range(2):                      # eager warm-up (sets kernel attributes)
-            for ph in phases:
+    tw = TimedWorkload(B, wl, layers, dev, stream, flags, arenas=2, temperature=args.temperature,
+                       no_graph=args.no_graph)
+    st = tw.st
+    if args.nvtx:
+        # named ranges around the four calls of one eager step, for a timeline tool
+        with torch.cuda.stream(stream):
+            for name, ph in zip(("diffusion_block_attend", "ar_verify_attend", "consensus_accept", "kv_append"),
+                                st.phases(0)):
+                torch.cuda.nvtx.range_push("orthrus_" + name)
                 ph()
-        stream.synchronize()
-        n0 = B.orthrus_launch_count()
-        for ph in phases:
-            ph()
-        launches_per_step = B.orthrus_launch_count() - n0
-        stream.synchronize()
-        graphs = None
-        if not args.no_graph:
-            graphs = [capture(ph, stream) for ph in phases]
+                torch.cuda.nvtx.range_pop()
+            stream.synchronize()
 
-        def step(events=None):
-            for i in range(4):
-                if events is not None:
-                    events[i].record(stream)
-                if graphs is not None:
-                    graphs[i].replay()
-                else:
-                    phases[i]()
-            if events is not None:
-                events[4].record(stream)
-
-        for _ in range(max(args.warmup, 3)):
-            step()
-        stream.synchronize()
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-        sampler = ClockSampler(local)
-        sampler.start()
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
-        for s in range(args.steps):
-            step(evs[s])
-        stream.synchronize()
-        torch.cuda.synchronize()
-        clocks = sampler.stop()
-        if dist is not None:
-            dist.barrier()
-
-        total_ms = evs[0][0].elapsed_time(evs[-1][4])
-        phase_ms = [statistics.mean(e[i].elapsed_time(e[i + 1]) for e in evs) for i in range(4)]
-        per_step = [e[0].elapsed_time(e[4]) for e in evs]
+    r = tw.run_timed(args.steps, args.warmup, args.min_region, local, dist)
+    phase_ms, per_step, clocks = r["phase_ms"], r["per_step"], r["clocks"]
+    with torch.cuda.stream(stream):
         read_probe = read_bandwidth_probe(dev, stream)
-        n_commit = st.n_commit.cpu()
-        status = B.orthrus_read_status(st.ws, stream)
-
-        # end-to-end arm: host buffers in, results out, every step
-        for _ in range(2):
-            st.h2d_inputs(); step(); st.d2h_results()
-        stream.synchronize()
-        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-        e2e_steps = max(3, min(args.steps, 20))
-        e0.record(stream)
-        for _ in range(e2e_steps):
-            h2d = st.h2d_inputs()
-            step()
-            d2h = st.d2h_results()
-        e1.record(stream)
-        stream.synchronize()
-        e2e_ms = e0.elapsed_time(e1) / e2e_steps
-
+    n_commit = st.n_commit.cpu()
+    status = B.orthrus_read_status(st.ws, stream)
+    e2e_steps = max(3, min(args.steps * r["inner"], 200))
+    e2e_serial_ms, h2d, d2h = tw.run_e2e(e2e_steps, overlap=False)
+    e2e_ms, h2d, d2h = tw.run_e2e(e2e_steps, overlap=True)
     if status != 0:
         raise SystemExit(f"bench.py: device status word {status} after the timed region")
 
-    ms_per_step = total_ms / args.steps
-    ms_per_step, e2e_ms = max_over_ranks([ms_per_step, e2e_ms], dist, dev)
+    ms_per_step, e2e_ms, e2e_serial_ms = max_over_ranks([r["ms_per_step"], e2e_ms, e2e_serial_ms], dist, dev)
 
     call_bytes = attend_bytes(wl, st.lens_host)
     step_bytes = call_bytes * 2 * layers
@@ -495,6 +634,9 @@ def run_gpu(args):
                    "prefix": [wl.prefix_min, wl.prefix_max], "vocab": wl.vocab, "layers": layers,
                    "step": "layers x (diffusion attend + AR verify attend) + consensus + "
                            "KV commit of all layers (+ rewind of cache_len)",
+                   "inner_repeats": r["inner"],
+                   "timed_region": f"{args.steps} steps x {r['inner']} back-to-back repetitions "
+                                   f"(at least {args.min_region} s), ms_per_step = region / (steps x repetitions)",
                    "l2": "inputs larger than L2 (distinct KV per layer)" if step_bytes > 2.5e8
                          else "L2-resident (reported, not a roofline workload)",
                    "cuda_graph": not args.no_graph, "attend_path": path,
@@ -517,13 +659,19 @@ def run_gpu(args):
         "tokens_per_forward_pass": round(tokens / wl.batch / 2.0, 4),
         "phase_ms": {"diffusion_attend": round(phase_ms[0], 5), "ar_verify_attend": round(phase_ms[1], 5),
                      "consensus": round(phase_ms[2], 5), "kv_commit": round(phase_ms[3], 5)},
-        "gpu_launches": int(launches_per_step * args.steps),
+        "gpu_launches": int(tw.launches_per_step * args.steps * r["inner"]),
         "clocks": clocks,
         "e2e": {"value": round(world * step_bytes / (e2e_ms * 1e-3) / 1e9, 2), "unit": "GB/s",
                 "ms_per_step": round(e2e_ms, 5), "h2d_bytes_per_step": int(h2d),
-                "d2h_bytes_per_step": int(d2h),
-                "note": "per-step inputs (Q, block KV, logits, drafts) from pinned host memory; "
-                        "the prefix KV cache is resident state"},
+                "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
+                "mode": "overlapped: two device arenas and a copy stream, the inputs of step s+1 cross "
+                        "the bus while step s computes",
+                "serial": {"value": round(world * step_bytes / (e2e_serial_ms * 1e-3) / 1e9, 2),
+                           "ms_per_step": round(e2e_serial_ms, 5),
+                           "mode": "copy in, compute, copy out on one stream"},
+                "note": "per-step inputs (Q, block KV of both views for every layer, logits, drafts) from "
+                        "pinned host memory; copied back: n_commit, committed, ar_argmax, next_anchor and the "
+                        "last layer's AR-view output; the prefix KV cache is resident state"},
         "roofline": {"bound": "hbm", "kernel": f"block attention ({path}) + split merge, per call",
                      "achieved": round(achieved, 2), "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": round(achieved / peak, 4),
@@ -535,12 +683,26 @@ def run_gpu(args):
         with torch.cuda.stream(stream):
             out["lm_head_consensus"] = lm_head_measure(B, wl, args.lm_head, dev, stream,
                                                        max(3, min(args.steps, 50)), local)
-    if args.decoder_cycles > 0:
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        out["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_budget, gpu_state=st)
+    tw.graphs = None
+    st.free()
+    del tw, st
+    torch.cuda.empty_cache()
+    if world == 1 and not args.no_extra_workloads and args.workload == DEFAULT_WORKLOAD and not args.block:
+        # the long-prefix and loop-shaped workloads on the same line: the bandwidth target is
+        # stated on these, the headline value stays the one above
+        out["workloads"] = {}
+        for name in ("cfg3_ragged", "cfg4_long", "cfg5_loop"):
+            out["workloads"][name] = workload_entry(B, name, dev, stream, flags, max(3, min(args.steps, 30)),
+                                                    local, peak)
+    cycles = args.decoder_cycles
+    if world == 1 and (cycles > 0 or (cycles == 0 and not args.no_extra_workloads and
+                                      args.workload == DEFAULT_WORKLOAD and not args.block)):
         with torch.cuda.stream(stream):
-            out["decoder_loop"] = decoder_loop_measure(B, dev, stream, args.decoder_cycles)
+            out["decoder_loop"] = decoder_loop_measure(B, dev, stream, 256 if cycles <= 0 else None,
+                                                       cycles if cycles > 0 else None)
     if rank == 0:
-        if not args.no_cpu_baseline and world == 1:
-            out["cpu_baseline"] = cpu_baseline(wl, budget_s=args.cpu_budget, gpu_state=st)
         print(json.dumps(out), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -639,114 +801,109 @@ def lm_head_measure(B, wl, hidden_dim, dev, stream, steps, gpu_index=0):
             "roofline": roof}
 
 
-def decoder_loop_measure(B, dev, stream, cycles):
-    """Whole generation cycles of a random-initialised decoder with the shapes of the
-    end-to-end configuration (12 layers, hidden 2048, 16/4 heads of 128, FFN 5632, vocabulary
-    32000, 8 sequences, prompts of 2048 tokens, block 16; about 1.2 GB of bf16 weights per
-    forward pass).  Everything off the hot path is plain torch (library GEMMs); both attention
-    passes, the LM-head-fused consensus and the commit go through the C ABI.  Drafts are forced
-    to agree with the AR view's precomputed greedy trajectory at a rate of 0.65 per position
-    (the diffusion view of a random-initialised model proposes nothing useful; once a sequence
-    leaves the precomputed trajectory at a near-tie its drafts stop agreeing), the diffusion
-    pass still runs in full.  One cycle is captured in a CUDA graph and replayed; the library's
-    share is the replay time of a second graph holding only that cycle's library calls."""
-    from harness.decoder import Decoder
+def decoder_loop_measure(B, dev, stream, n_new=256, max_cycles=None):
+    """The end-to-end configuration: a random-initialised decoder (12 layers, hidden 2048, 16/4
+    heads of 128, FFN 5632, vocabulary 32000, about 1.2 GB of bf16 weights per forward pass), 8
+    prompts of 2048 tokens, then `n_new` generated tokens per sequence by repeated block-16
+    draft / verify / consensus / commit.  Everything off the hot path is plain torch (library
+    GEMMs); both attention passes, the LM-head-fused consensus and the commit go through the
+    C ABI.  Drafts are forced: before every cycle an untimed width-1 look-ahead through the
+    same library calls gives the tokens greedy decoding emits next, and each draft copies its
+    look-ahead token with probability 0.65 (the diffusion view of a random-initialised model
+    proposes nothing useful; its pass still runs in full and is timed).  One cycle is captured
+    in a CUDA graph; every replay is bracketed by CUDA events and only the replays are timed.
+    The committed tokens are also compared with the look-ahead (the lossless property): a
+    mismatch is a near-tie that block verification and width-1 decoding round differently."""
+    from harness.decoder import Decoder, ForcedDraftLoop
     layers, hidden, n_q, n_kv, d, ffn, vocab = 12, 2048, 16, 4, 128, 5632, 32000
     Bt, T, K, rate = 8, 2048, 16, 0.65
-    n_traj = (cycles + 8) * K
-    cap = T + n_traj + 2 * K + 8
+    # room for the sequences that are ahead when the slowest one reaches its tokens
+    budget = (2 * n_new if n_new else max_cycles * K)
+    cap = T + budget + 4 * K + 8
     g = torch.Generator().manual_seed(W.sub_seed(W.BASE_SEED, "cfg5_loop", 0, "prompt"))
     prompt = torch.randint(0, vocab, (Bt, T), generator=g).to(dev)
     dec = Decoder(B, layers, hidden, n_q, n_kv, d, ffn, vocab, torch.bfloat16, Bt, cap, K, seed=5,
                   flags=B.LAYER_CACHE_QUIESCENT)
-    i32 = dict(dtype=torch.int32, device=dev)
-    head = dec.lm_head_rows()
     anchor0 = dec.prefill(prompt)
+    loop = ForcedDraftLoop(dec, anchor0, rate, seed=W.sub_seed(W.BASE_SEED, "cfg5_loop", 0, "draft"), fused=True)
     len0 = dec.cache_len.clone()
-    # the AR view's greedy trajectory (width-1 decoding), then rewind the cache length
-    outs1 = [torch.zeros(Bt, **i32), torch.zeros(Bt, 1, **i32), torch.zeros(Bt, 1, **i32), torch.zeros(Bt, **i32)]
-    ws1 = B.new_workspace(B.orthrus_lm_head_consensus_workspace_bytes(Bt, 1, vocab), device=dev)
-    zero1 = torch.zeros(Bt, 1, **i32)
-    traj, anchor = [], anchor0
-    for _ in range(n_traj):
-        _, ks, vs, hn = dec.forward_block(anchor.view(Bt, 1), "ar", 1, return_hidden=True, want_logits=False)
-        B.orthrus_lm_head_consensus(hn, head, zero1, *outs1, ws1)
-        dec.commit(ks, vs, outs1[0], 1)
-        anchor = outs1[3].clone()
-        traj.append(anchor)
-    traj = torch.stack(traj, 1)                                   # [B][n_traj]
-    dec.cache_len.copy_(len0)
-    wsK = B.new_workspace(B.orthrus_lm_head_consensus_workspace_bytes(Bt, K, vocab), device=dev)
-    done = torch.zeros(Bt, dtype=torch.int64, device=dev)
-    tokens = torch.zeros((), dtype=torch.int64, device=dev)
-    anchor = anchor0.clone()
-    ar = torch.arange(K, device=dev)
 
-    def cycle(record=None):
-        coin = torch.rand(Bt, K, device=dev) < rate
-        rnd = torch.randint(0, vocab, (Bt, K), device=dev, dtype=torch.int32)
-        idx = (done.view(Bt, 1) + ar).clamp(max=n_traj - 1)
-        draft = torch.where(coin, torch.gather(traj, 1, idx), rnd).to(torch.int32)
-        blk = torch.full((Bt, K), vocab, **i32)
-        blk[:, 0] = anchor
-        dec.forward_block(blk, "diff", K, want_logits=False, record=record)
-        ar_in = torch.cat([anchor.view(Bt, 1), draft[:, :K - 1]], dim=1)
-        _, ks, vs, hn = dec.forward_block(ar_in, "ar", K, return_hidden=True, want_logits=False, record=record)
-        tail = (lambda: (B.orthrus_lm_head_consensus(hn, head, draft, dec.n_commit, dec.committed, dec.ar_argmax,
-                                                     dec.next_anchor, wsK),
-                         dec.commit(ks, vs, dec.n_commit, K)))
-        tail()
-        if record is not None:
-            record.append(tail)
-        done.add_(dec.n_commit.long())
-        tokens.add_(dec.n_commit.sum())
-        anchor.copy_(dec.next_anchor)
-
-    for _ in range(3):
-        cycle()
+    # warm-up cycles (eager), then rewind: generation restarts from the prompt
+    for _ in range(2):
+        loop.lookahead(); loop.force_drafts(); loop.cycle()
     stream.synchronize()
+    dec.cache_len.copy_(len0); loop.anchor.copy_(anchor0); loop.done.zero_()
+    loop.lookahead(); loop.force_drafts()
     n0 = B.orthrus_launch_count()
     g_cycle = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g_cycle, stream=stream):
-        cycle()
+        loop.cycle()
     launches = B.orthrus_launch_count() - n0
+    # capture does not execute: state is still that of the prompt, drafts are in place
+
+    cycle_ms, tokens, mismatches, cycles = [], 0, 0, 0
+    evs = []
+    while True:
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        g_cycle.replay()
+        e1.record(stream)
+        evs.append((e0, e1))
+        n = dec.n_commit.cpu()
+        com, look = dec.committed.cpu(), loop.look.cpu()
+        for sq in range(Bt):
+            k = int(n[sq])
+            mismatches += int(not torch.equal(com[sq, :k], look[sq, :k]))
+        tokens += int(n.sum())
+        cycles += 1
+        if (n_new and int(loop.done.min()) >= n_new) or (max_cycles and cycles >= max_cycles):
+            break
+        if cycles > 4 * (n_new or 1 << 20):
+            raise SystemExit("bench.py: the decoder loop does not advance")
+        loop.lookahead(); loop.force_drafts()
+    stream.synchronize()
+    cycle_ms = [a.elapsed_time(b_) for a, b_ in evs]
+    total_ms = sum(cycle_ms)
+
+    # the library's share: the cycle's library calls alone, replayed from a graph of their own
     calls = []
-    cycle(calls)                                                  # eager, records the library calls
+    loop.lookahead(); loop.force_drafts()
+    loop.cycle(calls)
     stream.synchronize()
     len_mid = dec.cache_len.clone()
     g_lib = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g_lib, stream=stream):
         for f in calls:
             f()
-    dec.cache_len.copy_(len_mid)
-
-    def timed(graph, n, rewind):
-        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(n):
-            graph.replay()
-            if rewind:
-                dec.cache_len.copy_(len_mid)
-        e1.record(stream)
-        stream.synchronize()
-        return e0.elapsed_time(e1) / n
-
-    timed(g_lib, 3, True)
-    lib_ms = timed(g_lib, cycles, True)
-    timed(g_cycle, 2, False)
-    tokens.zero_()
-    ms = timed(g_cycle, cycles, False)
-    n_tok = int(tokens)
-    status = B.orthrus_read_status(dec.ws, stream) | B.orthrus_read_status(wsK, stream)
+    lib_n = 20
+    for it in range(3 + lib_n):
+        if it == 3:
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+        g_lib.replay()
+        dec.cache_len.copy_(len_mid)
+    e1.record(stream)
+    stream.synchronize()
+    lib_ms = e0.elapsed_time(e1) / lib_n
+    status = loop.status()
     if status != 0:
         raise SystemExit(f"bench.py: device status word {status} after the decoder loop")
-    return {"cycles": cycles, "ms_per_cycle": round(ms, 4),
-            "verified_tokens_per_s": round(n_tok / cycles / (ms * 1e-3), 1),
-            "verified_tokens_per_cycle": round(n_tok / cycles, 3),
-            "tokens_per_forward_pass": round(n_tok / cycles / Bt / 2.0, 4),
+    ms = total_ms / cycles
+    return {"generated_tokens_per_sequence": n_new, "cycles": cycles, "ms_per_cycle": round(ms, 4),
+            "ms_per_cycle_median": round(statistics.median(cycle_ms), 4),
+            "verified_tokens_per_s": round(tokens / (total_ms * 1e-3), 1),
+            "verified_tokens": tokens,
+            "verified_tokens_per_cycle": round(tokens / cycles, 3),
+            "tokens_per_forward_pass": round(tokens / cycles / Bt / 2.0, 4),
+            "near_tie_resyncs": mismatches,
+            "lossless_check": "committed tokens of every cycle compared with width-1 greedy decoding from the "
+                              "same state; a mismatch (counted above) ends that cycle's agreement and the "
+                              "reference restarts from the loop's own token",
             "in_library_ms_per_cycle": round(lib_ms, 4),
             "in_library_share": round(lib_ms / ms, 4),
             "library_launches_per_cycle": launches,
+            "timed": "CUDA-graph replays of whole cycles only; the look-ahead that forces the drafts is "
+                     "workload synthesis and runs between the timed replays",
             "model": {"layers": layers, "hidden": hidden, "q_heads": n_q, "kv_heads": n_kv, "head_dim": d,
                       "ffn": ffn, "vocab": vocab, "batch": Bt, "prompt": T, "block": K,
                       "forced_draft_agreement": rate, "weights": "random-initialised bf16",
@@ -890,8 +1047,13 @@ def main():
     ap.add_argument("--lm-head", type=int, default=0, metavar="HIDDEN",
                     help="also time the fused LM-head consensus at this hidden size (extra key)")
     ap.add_argument("--decoder-cycles", type=int, default=0, metavar="N",
-                    help="also time N whole generation cycles of the random-initialised decoder of the "
-                         "end-to-end configuration (extra key)")
+                    help="time N whole generation cycles of the random-initialised decoder of the end-to-end "
+                         "configuration instead of its 256 tokens per sequence (default run); -1: skip it")
+    ap.add_argument("--no-extra-workloads", action="store_true",
+                    help="only the headline workload: no `workloads` and no `decoder_loop` keys")
+    ap.add_argument("--min-region", type=float, default=0.5, metavar="SECONDS",
+                    help="every timed step is repeated back to back until the timed region lasts this long")
+    ap.add_argument("--nvtx", action="store_true", help="one eager step with NVTX ranges around the four calls")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-early-prefetch", action="store_true",
                     help="do not set ORTHRUS_LAYER_CACHE_QUIESCENT on the layers")

@@ -784,8 +784,9 @@ int tc_row_tiles(int G, int K)
 
 bool tc_driver_ok() { return encode_fn() != nullptr; }
 
-// CTAs of this kernel one SM of the current device keeps resident (2 on a B200: shared memory
-// binds); asked once per device, 2 assumed where there is no device to ask.
+// CTAs of this kernel one SM of the current device keeps resident: what its shared memory holds
+// (each CTA also costs the 1 KB the system reserves per block), at most the two that share
+// the 512 TMEM columns.  2 on a B200.  Asked once per device; 2 assumed where there is none.
 int tc_ctas_per_sm()
 {
     constexpr int kMaxDevices = 64;
@@ -795,12 +796,13 @@ int tc_ctas_per_sm()
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { (void)cudaGetLastError(); return 2; }
     std::lock_guard<std::mutex> lock(mu);
     if (cached[dev]) return cached[dev];
-    int n = 0;
-    if (cudaFuncSetAttribute(attend_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attend_tc_kernel<1>, NTHREADS, SMEM_BYTES) != cudaSuccess || n < 1) {
+    int smem_per_sm = 0;
+    if (cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess) {
         (void)cudaGetLastError();
         return 2;
     }
+    int n = smem_per_sm / (SMEM_BYTES + 1024);
+    n = n < 1 ? 1 : (n > 512 / (int)TM_COLS ? 512 / (int)TM_COLS : n);
     cached[dev] = n;
     return n;
 }
