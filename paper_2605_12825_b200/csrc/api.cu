@@ -166,10 +166,8 @@ static Plan make_plan(const orthrus_layer_t *L, bool tc)
 static size_t partial_bytes(const orthrus_layer_t *L, const Plan &pl, size_t *ml_off, bool tc = false)
 {
     if (ml_off) *ml_off = 0;
-    if (pl.n_splits == 1 ||
-        (tc && !tc_exchange_in_workspace(pl.n_splits, (L->n_q_heads / L->n_kv_heads) * L->block))) return 0;
-    // the tcgen05 path keeps one 128-row partial tile per CTA (exchanges too large for the
-    // on-chip path only)
+    if (pl.n_splits == 1) return 0;
+    // the tcgen05 path keeps one 128-row partial tile per CTA
     const size_t units = (size_t)L->batch * L->n_kv_heads *
                          (tc ? tc_row_tiles(L->n_q_heads / L->n_kv_heads, L->block) : 1);
     const size_t M = tc ? 128 : (size_t)(L->n_q_heads / L->n_kv_heads) * L->block;

@@ -23,18 +23,16 @@
 // bf16 operands carry without loss, and the result is the exact softmax because the
 // same shift is used for the numerator and the denominator.
 //
-// Narrow units (M <= 64) can optionally load their query rows twice and run two independent
-// softmax streams over the two column halves of every tile, so that all 128 softmax
-// threads work; the two streams are folded together in shared memory before the merge.
-//
-// Merge.  Every softmax thread puts its partial row (max, sum, unnormalised O straight out
-// of TMEM) into its CTA's idle ring.  Row r of the tile is merged and written by cluster
-// rank r % S.  Small exchanges (cluster size x rows < 1024) are read straight out of the
-// peers' shared memory, between two cluster barriers.  Larger ones go through the
-// workspace (L2): each CTA copies its rows out with 512-byte coalesced stores, one cluster
-// barrier publishes them, the owners read them back and a CTA leaves as soon as its own
-// rows are written; for those sizes the SM-to-SM path was measured to be slower.  There is
-// no second kernel.
+// Merge of the S partial results of a unit, inside the kernel (there is no second launch),
+// through the workspace, which stays in L2: every softmax thread stores its partial row (max, sum, unnormalised O) straight from the
+// registers its TMEM read-out filled, in a chunk-major layout ([16-byte column chunk][row])
+// so that a warp's 32 rows land in 512 contiguous bytes; one cluster barrier publishes the
+// rows; then the work is shared out as (32-row group, column chunk) tasks, one warp each,
+// round-robin over the cluster's CTAs and their warps: lane = row, all S partials of the
+// task are requested at once (again 512 contiguous bytes per request), weighted, summed,
+// normalised and written.  A CTA leaves as soon as its tasks are done.  (Reading the peers'
+// shared memory instead was measured slower at every cluster size: remote loads are round
+// trips with few requests in flight.)
 //
 // Programmatic dependent launch.  The kernel waits for the preceding kernel of the
 // stream (griddepcontrol.wait) before it reads anything that kernel may have written,
@@ -47,7 +45,9 @@
 // frees its TMEM and returns.
 #include <cuda.h>
 #include <cstdlib>
+#include <cstring>
 #include <mutex>
+#include <type_traits>
 #include <unordered_map>
 #include "common.cuh"
 #include "tc_ptx.cuh"
@@ -67,12 +67,9 @@ constexpr int SLOT_BYTES = 2 * SUB_BYTES;
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int OFF_Q = 0;                                   // [128][128] bf16, 2 sub-tiles
 constexpr int OFF_RING = OFF_Q + 2 * QSUB_BYTES;           // NSLOT x 16 KB
-constexpr int OFF_OPART = OFF_RING;                        // float [128][128], after the last MMA
-constexpr int OFF_ML = OFF_OPART + MROWS * HD * 4;         // float [128][2], inside the ring
 constexpr int OFF_BAR = OFF_RING + NSLOT * SLOT_BYTES;     // mbarriers
 constexpr int OFF_MISC = OFF_BAR + 24 * 8;                 // tmem base, abort flag, unit
 constexpr int SMEM_BYTES = OFF_MISC + 64;
-static_assert(OFF_ML + MROWS * 8 <= OFF_BAR, "partial rows must fit in the idle ring");
 static_assert(2 * (SMEM_BYTES + 1024) <= 228 * 1024, "two CTAs per SM");
 
 enum { BAR_FULL = 0, BAR_EMPTY = NSLOT, BAR_QFULL = 2 * NSLOT, BAR_SFULL, BAR_PFULL = BAR_SFULL + 2,
@@ -81,115 +78,66 @@ static_assert(NUM_BARS <= 24, "barrier area");
 
 constexpr uint32_t TM_O = 0, TM_S = 128, TM_COLS = 256;   // TMEM column map
 constexpr float RESCALE_THRESHOLD = 8.f;                  // log2 units
-// a cluster whose partial rows add up to this many (cluster size x rows per CTA) or more
-// exchanges them through the L2 workspace instead of distributed shared memory
-constexpr int kL2ExchangeRows = 1024;
-
 struct TcMaps { CUtensorMap k, v, q, kb, vb; };
 
-// Split merge.  Row R of a tile is merged and written by cluster rank R % S: a warp per row,
-// lane j holds the weight of the partial result of rank j, every lane four output columns.
-// load_ml(j, R) returns (max, sum) of rank j's partial row R, load_o(j, R) this lane's four
-// columns of it.  The loads of a batch are all issued before the first is used.
-template <class LoadML, class LoadO, class Store>
-__device__ inline void merge_rows(int S, int rank, int my_rows, int warp, int lane, int n_warps,
-                                  LoadML load_ml, LoadO load_o, Store store)
+// Merge through the workspace.  A task is (32-row group, 16-byte column chunk) of a unit; lane =
+// row of the group.  Tasks go round-robin to the cluster's CTAs and their warps.  A warp takes
+// 16 / SP tasks per round (SP = cluster size rounded up to a power of two), so that sixteen
+// 16-byte loads per lane are in flight whatever the cluster size; every load of a warp covers
+// 512 contiguous bytes.  grp_o: the cluster's S partial tiles, each [32 chunks][128 rows] of
+// float4; grp_ml: (max, sum) per [CTA][row].  store(R, chunk, acc, 1 / sum).
+template <int SP, class Store>
+__device__ inline void l2_merge_tasks(int S, int rank, int warp, int lane, int n_warps, int n_tasks, int rows_here,
+                                      const float4 *grp_o, const float2 *grp_ml, Store store)
 {
-    if (my_rows <= n_warps) {
-        // at most one row per warp: all of the row's partial results are requested at once
-        if (warp < my_rows) {
-            const int R = rank + warp * S;
-            float mj = -INFINITY, lj = 0.f;
-            if (lane < S) { const float2 t2 = load_ml(lane, R); mj = t2.x; lj = t2.y; }
-            float4 v[16];
+    constexpr int TB = 16 / SP;
+    // task index of (round, slot u) for this warp: consecutive tasks of a round sit S * n_warps apart
+    for (int t0 = rank + warp * S; t0 < n_tasks; t0 += S * n_warps * TB) {
+        float2 ml[TB][SP];
+        float4 o[TB][SP];
 #pragma unroll
-            for (int u = 0; u < 16; ++u)
-                if (u < S) v[u] = load_o(u, R);
-            float mmax = mj;
+        for (int u = 0; u < TB; ++u) {
+            const int task = t0 + u * S * n_warps;
+            const int R = (task / (HD / 4)) * 32 + lane, c = task % (HD / 4);
+            const bool live = task < n_tasks && R < rows_here;
 #pragma unroll
-            for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
-            const float wj = (lj > 0.f) ? ex2(mj - mmax) : 0.f;
-            float L = wj * lj;
-#pragma unroll
-            for (int off = 16; off; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int u = 0; u < 16; ++u) {
-                const float w = (u < S) ? __shfl_sync(0xffffffffu, wj, u) : 0.f;
-                // a partial without keys has weight 0 and its row was never written
-                if (w != 0.f) {
-                    acc.x = fmaf(w, v[u].x, acc.x); acc.y = fmaf(w, v[u].y, acc.y);
-                    acc.z = fmaf(w, v[u].z, acc.z); acc.w = fmaf(w, v[u].w, acc.w);
+            for (int j = 0; j < SP; ++j)
+                if (j < S && live) {
+                    ml[u][j] = __ldcg(grp_ml + j * MROWS + R);
+                    o[u][j] = __ldcg(grp_o + (long long)j * (MROWS * HD / 4) + c * MROWS + R);
                 }
-            }
-            store(R, acc, 1.f / L);
         }
-        return;
-    }
-    for (int s0 = warp; s0 < my_rows; s0 += 4 * n_warps) {
-        float mj[4], lj[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int R = rank + min(s0 + q * n_warps, my_rows - 1) * S;
-            mj[q] = -INFINITY; lj[q] = 0.f;
-            if (lane < S && s0 + q * n_warps < my_rows) { const float2 t2 = load_ml(lane, R); mj[q] = t2.x; lj[q] = t2.y; }
-        }
-        float4 acc[4];
+        for (int u = 0; u < TB; ++u) {
+            const int task = t0 + u * S * n_warps;
+            const int R = (task / (HD / 4)) * 32 + lane, c = task % (HD / 4);
+            if (task < n_tasks && R < rows_here) {
+                float mmax = -INFINITY;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        float wj[4] = {0.f, 0.f, 0.f, 0.f}, L[4] = {1.f, 1.f, 1.f, 1.f};
-        for (int j0 = 0; j0 < S; j0 += 4) {
-            float4 v[4][4];
+                for (int j = 0; j < SP; ++j)
+                    if (j < S && ml[u][j].y > 0.f) mmax = fmaxf(mmax, ml[u][j].x);
+                float L = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int R = rank + min(s0 + q * n_warps, my_rows - 1) * S;
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (j0 + u < S && s0 + q * n_warps < my_rows) v[q][u] = load_o(j0 + u, R);
-            }
-            if (j0 == 0) {
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    float mmax = mj[q];
-#pragma unroll
-                    for (int off = 16; off; off >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, off));
-                    wj[q] = (lj[q] > 0.f) ? ex2(mj[q] - mmax) : 0.f;
-                    L[q] = wj[q] * lj[q];
-#pragma unroll
-                    for (int off = 16; off; off >>= 1) L[q] += __shfl_xor_sync(0xffffffffu, L[q], off);
-                }
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const float w = (j0 + u < S) ? __shfl_sync(0xffffffffu, wj[q], min(j0 + u, 31)) : 0.f;
-                    // a partial without keys has weight 0 and its row was never written
-                    if (w != 0.f) {
-                        acc[q].x = fmaf(w, v[q][u].x, acc[q].x); acc[q].y = fmaf(w, v[q][u].y, acc[q].y);
-                        acc[q].z = fmaf(w, v[q][u].z, acc[q].z); acc[q].w = fmaf(w, v[q][u].w, acc[q].w);
+                for (int j = 0; j < SP; ++j)
+                    if (j < S && ml[u][j].y > 0.f) {      // a partial without keys was never written
+                        const float w = ex2(ml[u][j].x - mmax);
+                        L = fmaf(w, ml[u][j].y, L);
+                        acc.x = fmaf(w, o[u][j].x, acc.x); acc.y = fmaf(w, o[u][j].y, acc.y);
+                        acc.z = fmaf(w, o[u][j].z, acc.z); acc.w = fmaf(w, o[u][j].w, acc.w);
                     }
-                }
+                store(R, c, acc, 1.f / L);
+            }
         }
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-            if (s0 + q * n_warps < my_rows) store(rank + (s0 + q * n_warps) * S, acc[q], 1.f / L[q]);
     }
 }
 
-// NSUB = 1: thread r of the softmax warps owns query row r and all 64 columns of a tile.
-// NSUB = 2 (units of at most 64 rows): the query rows are loaded twice, rows 64..127 being a
-// copy of rows 0..63; thread r works on logical row r % 64 and on columns [32*(r/64), +32)
-// of every tile only, so all 128 threads have work.  The two halves are independent
-// online-softmax streams (own max, own sum, own O row in TMEM) that are folded together
-// at the end exactly like the partial results of different CTAs.
-template <int NSUB>
+// Thread r of the softmax warps owns query row r (TMEM lane r) and all 64 columns of a tile.
 __global__ void __launch_bounds__(NTHREADS, 2)
 attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const int S, const int kb_rows,
                  const int quiescent)
 {
-    constexpr int W = TN / NSUB;              // score columns per softmax thread
-    constexpr int MPAD = MROWS / NSUB;        // logical rows per sub-stream
+    constexpr int W = TN;                     // score columns per softmax thread
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t sbase = smem_u32(smem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + OFF_MISC + 8);
@@ -200,10 +148,10 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int rank = S > 1 ? (int)cluster_rank() : 0;
     const int order = blockIdx.y, rt = blockIdx.z;
-    // this row tile: kb_rows block positions x G heads (at most MPAD rows)
+    // this row tile: kb_rows block positions x G heads (at most 128 rows)
     const int i0 = rt * kb_rows;
     const int rows_here = min(p.K - i0, kb_rows) * p.G;
-    const int n_act = NSUB * ((rows_here + 31) >> 5);         // softmax warps with rows
+    const int n_act = (rows_here + 31) >> 5;                  // softmax warps with rows
     const bool aligned = (sbase & 1023u) == 0;                // swizzled tiles need 1 KB alignment
 
     // ------------------------------------------------------------------ prologue
@@ -305,11 +253,9 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
 
     if (warp < 4) {
         const int r = tid;
-        const int sub = r / MPAD, Rl = r % MPAD;              // sub-stream, logical row in the tile
-        const bool valid = Rl < rows_here;
-        const bool warp_active = ((warp * 32) % MPAD) < rows_here;
-        const int i_row = i0 + Rl / p.G;
-        const int col0 = sub * W;
+        const bool valid = r < rows_here;
+        const bool warp_active = warp * 32 < rows_here;
+        const int i_row = i0 + r / p.G;
         const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
         float m_run = -INFINITY, l_run = 0.f;
         bool have_o = false;
@@ -325,13 +271,13 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                 tc_fence_after();
                 uint32_t s[W];
 #pragma unroll
-                for (int c = 0; c < W / 32; ++c) tmem_ld32(lane_base + TM_S + sb * TN + col0 + c * 32, s + c * 32);
+                for (int c = 0; c < W / 32; ++c) tmem_ld32(lane_base + TM_S + sb * TN + c * 32, s + c * 32);
                 tmem_ld_wait();
-                // visible columns of this row in this tile, then in this thread's column range
+                // visible columns of this row in this tile
                 int lim;
                 if (t < n_mine) lim = min(TN, P - ((int)t0 + t) * TN);
                 else lim = p.causal ? min(p.K, i_row + 1) : p.K;
-                lim = valid ? min(W, max(0, lim - col0)) : 0;
+                lim = valid ? lim : 0;
                 float mx;
                 if (lim == W) {
                     float m4[4];
@@ -413,17 +359,8 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                     }
                 }
                 l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
-                // P over the scores, 2 bf16 per column: the row's 32 packed columns are this
-                // thread's range and zeros for the range of the other sub-stream
-                if constexpr (NSUB == 1) {
-                    tmem_st32(lane_base + TM_S + sb * TN, pk);
-                } else {
-                    uint32_t zero[16];
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) zero[j] = 0u;
-                    tmem_st16(lane_base + TM_S + sb * TN + sub * 16, pk);
-                    tmem_st16(lane_base + TM_S + sb * TN + (1 - sub) * 16, zero);
-                }
+                // P over the scores, 2 bf16 per 32-bit column
+                tmem_st32(lane_base + TM_S + sb * TN, pk);
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
@@ -436,13 +373,13 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             have_o = ok;
         }
 
-        if (S == 1 && NSUB == 1) {
+        if (S == 1) {
             // ---------------------------------------------------------- direct output
             // the whole unit was here: normalise and write the final rows
             if (have_o) {
                 const float inv = 1.f / l_run;
                 __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(p.out) +
-                    (((long long)b * p.K + i_row) * p.Hq + h * p.G + (Rl % p.G)) * HD;
+                    (((long long)b * p.K + i_row) * p.Hq + h * p.G + (r % p.G)) * HD;
 #pragma unroll 1
                 for (int c4 = 0; c4 < HD / 32; ++c4) {
                     uint32_t o[32];
@@ -462,78 +399,37 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                 }
             }
         } else {
-            // ---------------------------------------------------------- publish partial rows
-            // every softmax thread puts its partial row (max, sum, unnormalised O straight out
-            // of TMEM) into this CTA's ring, which is idle once the last product has retired
+            // ---------------------------------------------------------- partial rows to the workspace
+            // straight from the registers of the TMEM read-out: element (chunk c, row r) of this
+            // CTA's [32 chunks][128 rows] array of 16-byte chunks, so a warp stores 512 contiguous bytes
+            const long long cta_lin = ((long long)rt * gridDim.y + order) * S + rank;
+            float4 *my_o = reinterpret_cast<float4 *>(p.part_o + cta_lin * (MROWS * HD));
+            float2 *my_ml = reinterpret_cast<float2 *>(p.part_ml + cta_lin * (MROWS * 2));
             if (have_o) {
-#pragma unroll 1
-                for (int c2 = 0; c2 < HD / 64; ++c2) {
-                    uint32_t o[64];
-                    tmem_ld32(lane_base + TM_O + c2 * 64, o);
-                    tmem_ld32(lane_base + TM_O + c2 * 64 + 32, o + 32);
-                    tmem_ld_wait();
+                // the whole row in one read-out (one wait instead of four), then 32 stores
+                uint32_t o[HD];
 #pragma unroll
-                    for (int c = 0; c < 16; ++c)
-                        *reinterpret_cast<uint4 *>(smem + OFF_OPART + r * 512 + (((c2 * 16 + c) ^ (r & 31)) << 4)) =
-                            make_uint4(o[c * 4], o[c * 4 + 1], o[c * 4 + 2], o[c * 4 + 3]);
+                for (int c4 = 0; c4 < HD / 32; ++c4) tmem_ld32(lane_base + TM_O + c4 * 32, o + c4 * 32);
+                tmem_ld_wait();
+                if (valid) {
+#pragma unroll
+                    for (int c = 0; c < HD / 4; ++c)
+                        __stcg(my_o + c * MROWS + r,
+                               make_float4(__uint_as_float(o[c * 4]), __uint_as_float(o[c * 4 + 1]),
+                                           __uint_as_float(o[c * 4 + 2]), __uint_as_float(o[c * 4 + 3])));
                 }
             }
-            if (valid && (have_o || !active)) {   // (threads without a row may get here before the ring is idle)
-                float *ml = reinterpret_cast<float *>(smem + OFF_ML);
-                ml[r * 2] = have_o ? m_run : -INFINITY;       // a CTA without tiles has empty rows
-                ml[r * 2 + 1] = have_o ? l_run : 0.f;
-            }
-            if constexpr (NSUB == 2) {
-                // fold the two sub-streams of a row together, in place in the first one's row:
-                // a warp per logical row, lane c holds output columns 4c..4c+3
-                named_bar_sync(1, 128);
-                float *ml = reinterpret_cast<float *>(smem + OFF_ML);
-                for (int R0 = warp; R0 < rows_here; R0 += 16) {   // four rows at a time, for latency
-                    float2 ma[4], mb[4];
-                    float4 va[4], vb[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int R = min(R0 + 4 * q, rows_here - 1), R2 = R + MPAD;
-                        ma[q] = *reinterpret_cast<const float2 *>(ml + R * 2);
-                        mb[q] = *reinterpret_cast<const float2 *>(ml + R2 * 2);
-                        va[q] = *reinterpret_cast<const float4 *>(smem + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4));
-                        vb[q] = *reinterpret_cast<const float4 *>(smem + OFF_OPART + R2 * 512 + ((lane ^ (R2 & 31)) << 4));
-                    }
-                    __syncwarp();
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int R = R0 + 4 * q;
-                        if (R < rows_here) {
-                            // a sub-stream without keys has sum 0 and its row was never written
-                            const bool ha = ma[q].y > 0.f, hb = mb[q].y > 0.f;
-                            const float mm = fmaxf(ha ? ma[q].x : -INFINITY, hb ? mb[q].x : -INFINITY);
-                            const float wa = ha ? ex2(ma[q].x - mm) : 0.f, wb = hb ? ex2(mb[q].x - mm) : 0.f;
-                            float4 o;
-                            o.x = wa * (ha ? va[q].x : 0.f) + wb * (hb ? vb[q].x : 0.f);
-                            o.y = wa * (ha ? va[q].y : 0.f) + wb * (hb ? vb[q].y : 0.f);
-                            o.z = wa * (ha ? va[q].z : 0.f) + wb * (hb ? vb[q].z : 0.f);
-                            o.w = wa * (ha ? va[q].w : 0.f) + wb * (hb ? vb[q].w : 0.f);
-                            *reinterpret_cast<float4 *>(smem + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4)) = o;
-                            if (lane == 0)
-                                *reinterpret_cast<float2 *>(ml + R * 2) =
-                                    make_float2(mm, wa * ma[q].y + wb * mb[q].y);
-                        }
-                    }
-                }
-            }
+            // (a CTA without tiles has empty rows: sum 0, and its O rows are never read)
+            if (valid) __stcg(my_ml + r, make_float2(have_o ? m_run : -INFINITY, have_o ? l_run : 0.f));
         }
         tc_fence_before();
     } else if (warp == 4) {
         // ------------------------------------------------------------------ producer
         if (active && lane == 0) {
-            // the query rows of this tile: box = 64 columns x G heads x kb_rows positions,
-            // once per sub-stream
-            mbar_expect_tx(bar(BAR_QFULL), (uint32_t)(NSUB * 2 * 128 * p.G * kb_rows));
-#pragma unroll
-            for (int u = 0; u < NSUB; ++u) {
-                tma_load_4d(sbase + OFF_Q + u * MPAD * 128, &tm.q, 0, h * p.G, i0, b, bar(BAR_QFULL));
-                tma_load_4d(sbase + OFF_Q + QSUB_BYTES + u * MPAD * 128, &tm.q, 64, h * p.G, i0, b, bar(BAR_QFULL));
-            }
+            // the query rows of this tile: box = 64 columns x G heads x kb_rows positions
+            mbar_expect_tx(bar(BAR_QFULL), (uint32_t)(2 * 128 * p.G * kb_rows));
+            tma_load_4d(sbase + OFF_Q, &tm.q, 0, h * p.G, i0, b, bar(BAR_QFULL));
+            tma_load_4d(sbase + OFF_Q + QSUB_BYTES, &tm.q, 64, h * p.G, i0, b, bar(BAR_QFULL));
             bool ok = true;
             const int n_items = 2 * n_tiles;
             while (produced < n_items && ok) {
@@ -623,75 +519,32 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     if (warp == 5)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TM_COLS) : "memory");
     if (tid == 0 && *abort_flag && p.status) atomicOr(p.status, ORTHRUS_DEV_WAIT_TIMEOUT);
-    if (S == 1 && NSUB == 1) return;
+    if (S == 1) return;
     constexpr int NWARPS = NTHREADS / 32;
-    if (S == 1) {
-        // the two sub-streams of a lone CTA were folded in shared memory: normalise and write
-        const float *ml = reinterpret_cast<const float *>(smem + OFF_ML);
-        for (int R = warp; R < rows_here; R += NWARPS) {
-            const float4 v = *reinterpret_cast<const float4 *>(smem + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4));
-            const float inv = 1.f / ml[R * 2 + 1];
-            const int i = i0 + R / p.G, g = R % p.G;
-            uint2 *dst = reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) +
-                         (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD);
-            dst[lane] = make_uint2(pack_bf16(v.x * inv, v.y * inv), pack_bf16(v.z * inv, v.w * inv));
-        }
-        return;
-    }
-
-    // How the CTAs of a cluster exchange their partial rows.  Small exchanges: each CTA reads
-    // the rows it merges straight out of its peers' shared memory.  Large ones (cluster size x
-    // rows >= 1024, e.g. 16 CTAs x 64 rows or 8 x 128): through the workspace, which lives in
-    // L2; an all-to-all of that size over the SM-to-SM path moved about 5 bytes per cycle per
-    // SM and took longer than the whole stream of keys.  The cluster is what guarantees that
-    // the CTAs waiting for one another are resident together.
-    const int my_rows = rank < rows_here ? (rows_here - rank + S - 1) / S : 0;
-    auto store = [&](int R, const float4 &acc, float inv) {
+    auto out_row = [&](int R) {
         const int i = i0 + R / p.G, g = R % p.G;
-        uint2 *dst = reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(p.out) +
-                     (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD);
-        dst[lane] = make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+        return static_cast<__nv_bfloat16 *>(p.out) + (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD;
     };
-    if (S * rows_here >= kL2ExchangeRows) {
-        const long long cta_lin = ((long long)rt * gridDim.y + order) * S + rank;
-        float *my_o = p.part_o + cta_lin * (MROWS * HD);
-        float *my_ml = p.part_ml + cta_lin * (MROWS * 2);
-        const float *ml = reinterpret_cast<const float *>(smem + OFF_ML);
-        // copy this CTA's rows out: a warp per row, 512 contiguous bytes
-        for (int R0 = warp; R0 < rows_here; R0 += 4 * NWARPS) {
-            float4 v[4];
-            float2 t2[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int R = min(R0 + q * NWARPS, rows_here - 1);
-                v[q] = *reinterpret_cast<const float4 *>(smem + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4));
-                t2[q] = *reinterpret_cast<const float2 *>(ml + R * 2);
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int R = R0 + q * NWARPS;
-                if (R < rows_here) {
-                    // (the row of a CTA without keys was never written: only its sum 0 matters)
-                    reinterpret_cast<float4 *>(my_o + R * HD)[lane] = v[q];
-                    if (lane == 0) *reinterpret_cast<float2 *>(my_ml + R * 2) = t2[q];
-                }
-            }
-        }
-        cluster_sync_all();               // release / acquire at cluster scope: the rows are in place
-        const float *grp_o = p.part_o + (cta_lin - rank) * (MROWS * HD);
-        const float *grp_ml = p.part_ml + (cta_lin - rank) * (MROWS * 2);
-        merge_rows(S, rank, my_rows, warp, lane, NWARPS,
-                   [&](int j, int R) { return __ldcg(reinterpret_cast<const float2 *>(grp_ml + (long long)j * (MROWS * 2) + R * 2)); },
-                   [&](int j, int R) { return __ldcg(reinterpret_cast<const float4 *>(grp_o + (long long)j * (MROWS * HD) + R * HD) + lane); },
-                   store);
-        return;                           // nobody reads this CTA's shared memory
+    {
+        // The cluster is what guarantees that the CTAs waiting for one another are resident
+        // together.  Release / acquire at cluster scope: every CTA's partial rows are in place.
+        cluster_sync_all();
+        const long long grp_lin = ((long long)rt * gridDim.y + order) * S;
+        const float4 *grp_o = reinterpret_cast<const float4 *>(p.part_o + grp_lin * (MROWS * HD));
+        const float2 *grp_ml = reinterpret_cast<const float2 *>(p.part_ml + grp_lin * (MROWS * 2));
+        const int n_tasks = ((rows_here + 31) >> 5) * (HD / 4);
+        auto run = [&](auto sp) {
+            l2_merge_tasks<decltype(sp)::value>(S, rank, warp, lane, NWARPS, n_tasks, rows_here, grp_o, grp_ml,
+                                                [&](int R, int c, const float4 &acc, float inv) {
+                reinterpret_cast<uint2 *>(out_row(R))[c] =
+                    make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+            });
+        };
+        if (S <= 2) run(std::integral_constant<int, 2>());
+        else if (S <= 4) run(std::integral_constant<int, 4>());
+        else if (S <= 8) run(std::integral_constant<int, 8>());
+        else run(std::integral_constant<int, 16>());
     }
-    cluster_sync_all();                   // every CTA's partial rows are in place
-    merge_rows(S, rank, my_rows, warp, lane, NWARPS,
-               [&](int j, int R) { return ld_cluster_f2(map_to_rank(sbase + OFF_ML + R * 8, j)); },
-               [&](int j, int R) { return ld_cluster_f4(map_to_rank(sbase + OFF_OPART + R * 512 + ((lane ^ (R & 31)) << 4), j)); },
-               store);
-    cluster_sync_all();                   // peers may still be reading this CTA's rows
 }
 
 // ---------------------------------------------------------------------------- host side
@@ -763,22 +616,13 @@ bool get_map(const void *ptr, unsigned long long d1, unsigned long long d2, unsi
 
 }  // namespace
 
-// Sub-streams per query row: 2 when a unit has at most 64 rows, else 1.
-// Sub-streams per query row.  Two sub-streams halve the softmax time of a tile for units of
-// at most 64 rows, but their extra fold step costs more than that at the tile counts per
-// CTA measured so far, so they are opt-in (ORTHRUS_TC_NSUB=2) and one is the default.
-static int tc_nsub(int G, int K)
-{
-    static const int forced = [] { const char *e = getenv("ORTHRUS_TC_NSUB"); return e ? atoi(e) : 0; }();
-    return (forced == 2 && G * K <= 64) ? 2 : 1;
-}
-// block positions per query tile of 128 / nsub rows
-static int tc_kb_rows(int G, int K, int nsub) { return K < (MROWS / nsub) / G ? K : (MROWS / nsub) / G; }
+// block positions per query tile of 128 rows
+static int tc_kb_rows(int G, int K) { return K < MROWS / G ? K : MROWS / G; }
 
 int tc_row_tiles(int G, int K)
 {
     if (G < 1 || G > MROWS) return 0;
-    const int kb = tc_kb_rows(G, K, tc_nsub(G, K));
+    const int kb = tc_kb_rows(G, K);
     return (K + kb - 1) / kb;
 }
 
@@ -820,8 +664,8 @@ int tc_max_cluster()
     std::lock_guard<std::mutex> lock(mu);
     if (cached[dev]) return cached[dev];
     int best = 16;
-    if (cudaFuncSetAttribute(attend_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
-        cudaFuncSetAttribute(attend_tc_kernel<1>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+    if (cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
+        cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
         for (int s = 16; s >= 2; s >>= 1) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(s, 1, 1);
@@ -832,7 +676,7 @@ int tc_max_cluster()
             attr[0].val.clusterDim.x = s; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
             cfg.attrs = attr; cfg.numAttrs = 1;
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, attend_tc_kernel<1>, &cfg) == cudaSuccess && n > 0) { best = s; break; }
+            if (cudaOccupancyMaxActiveClusters(&n, attend_tc_kernel, &cfg) == cudaSuccess && n > 0) { best = s; break; }
             best = s >> 1;
         }
         if (best < 1) best = 1;
@@ -843,9 +687,6 @@ int tc_max_cluster()
     return best;
 }
 int tc_tile_positions() { return TN; }
-bool tc_exchange_in_workspace(int S, int M) { return S * (M < MROWS ? M : MROWS) >= kL2ExchangeRows; }
-
-template <int NSUB>
 static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int flags, cudaStream_t st)
 {
     const int S = p.n_splits;
@@ -859,9 +700,9 @@ static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int 
         if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
         std::lock_guard<std::mutex> lock(mu);
         if (!configured[dev]) {
-            e = cudaFuncSetAttribute(attend_tc_kernel<NSUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+            e = cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
             if (e == cudaSuccess)
-                e = cudaFuncSetAttribute(attend_tc_kernel<NSUB>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+                e = cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
             if (e != cudaSuccess) return e;
             configured[dev] = true;
         }
@@ -887,7 +728,7 @@ static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int 
     }
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, attend_tc_kernel<NSUB>, p, tm, S, kb,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attend_tc_kernel, p, tm, S, kb,
                                        (flags & ORTHRUS_LAYER_CACHE_QUIESCENT) ? 1 : 0);
     count_launch();
     return e;
@@ -895,15 +736,14 @@ static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int 
 
 cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st)
 {
-    const int nsub = tc_nsub(p.G, p.K);
-    const int kb = tc_kb_rows(p.G, p.K, nsub);
+    const int kb = tc_kb_rows(p.G, p.K);
     TcMaps tm;
     const unsigned long long rows = (unsigned long long)p.B * p.Hkv * p.capacity;
     if (!get_map(p.k_cache, rows, 0, 0, TN, 0, &tm.k) || !get_map(p.v_cache, rows, 0, 0, TN, 0, &tm.v) ||
         !get_map(p.q, p.Hq, p.K, p.B, p.G, kb, &tm.q) ||
         !get_map(p.k_blk, p.Hkv, p.K, p.B, 1, TN, &tm.kb) || !get_map(p.v_blk, p.Hkv, p.K, p.B, 1, TN, &tm.vb))
         return cudaErrorInvalidValue;
-    return nsub == 2 ? launch_tc<2>(p, tm, kb, flags, st) : launch_tc<1>(p, tm, kb, flags, st);
+    return launch_tc(p, tm, kb, flags, st);
 }
 
 }  // namespace orthrus

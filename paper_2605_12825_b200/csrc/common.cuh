@@ -71,7 +71,6 @@ int tc_row_tiles(int G, int K);          // 128-row query tiles per unit (0: gro
 int tc_ctas_per_sm();
 int tc_max_cluster();                   // largest cluster the device can co-schedule (<= 16)
 int tc_tile_positions();
-bool tc_exchange_in_workspace(int S, int M);   // split partials of S CTAs x M rows go through the workspace
 cudaError_t launch_combine(const AttnParams &p, int dtype, cudaStream_t st);
 
 cudaError_t launch_consensus(const void *logits, int dtype, const int32_t *draft, int B, int K,
