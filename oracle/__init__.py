@@ -100,15 +100,17 @@ def _check(t: torch.Tensor, name: str) -> torch.Tensor:
 
 
 def _desc(q, k_blk, v_blk, k_cache, v_cache, cache_len, scale) -> _AttnDesc:
+    """k_blk = v_blk = None: the block's K/V rows are the cache rows [P_b, P_b + K)."""
     B, K, Hq, d = q.shape
     Hkv, cap = k_cache.shape[1], k_cache.shape[2]
     dt = q.dtype
-    for n, t in (("q", q), ("k_blk", k_blk), ("v_blk", v_blk),
-                 ("k_cache", k_cache), ("v_cache", v_cache)):
+    in_cache = k_blk is None and v_blk is None
+    for n, t in (("q", q), ("k_cache", k_cache), ("v_cache", v_cache)) + \
+            (() if in_cache else (("k_blk", k_blk), ("v_blk", v_blk))):
         _check(t, n)
         if t.dtype != dt:
             raise ValueError("all attention tensors must share one dtype")
-    if tuple(k_blk.shape) != (B, K, Hkv, d) or tuple(v_blk.shape) != (B, K, Hkv, d):
+    if not in_cache and (tuple(k_blk.shape) != (B, K, Hkv, d) or tuple(v_blk.shape) != (B, K, Hkv, d)):
         raise ValueError("block KV must be [B][K][Hkv][d]")
     if tuple(k_cache.shape) != (B, Hkv, cap, d) or tuple(v_cache.shape) != (B, Hkv, cap, d):
         raise ValueError("cache must be [B][Hkv][capacity][d]")
@@ -116,7 +118,8 @@ def _desc(q, k_blk, v_blk, k_cache, v_cache, cache_len, scale) -> _AttnDesc:
     if cache_len.dtype != torch.int32 or cache_len.numel() != B:
         raise ValueError("cache_len must be int32 [B]")
     return _AttnDesc(B, K, Hq, Hkv, d, _DTYPE_CODE[dt], cap,
-                     q.data_ptr(), k_blk.data_ptr(), v_blk.data_ptr(),
+                     q.data_ptr(), None if in_cache else k_blk.data_ptr(),
+                     None if in_cache else v_blk.data_ptr(),
                      k_cache.data_ptr(), v_cache.data_ptr(), cache_len.data_ptr(),
                      float(scale) if scale else 0.0)
 
@@ -274,3 +277,44 @@ def kv_append(k_cache, v_cache, cache_len, k_blk, v_blk, n_commit, update_len: b
                                       cache_len.data_ptr(), k_blk.data_ptr(),
                                       v_blk.data_ptr(), n_commit.data_ptr(),
                                       1 if update_len else 0))
+
+
+def block_kv_write(k_cache, v_cache, cache_len, k_blk, v_blk) -> int:
+    """Step 1 of the write-then-truncate commit: all K block rows go behind the prefix, the
+    length stays.  In place; returns the C status (0, or -3 if a sequence lacked room)."""
+    for n_, t in (("k_cache", k_cache), ("v_cache", v_cache), ("cache_len", cache_len),
+                  ("k_blk", k_blk), ("v_blk", v_blk)):
+        _check(t, n_)
+    B, Hkv, cap, d = k_cache.shape
+    K = k_blk.shape[1]
+    f = lib().oracle_block_kv_write
+    f.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64,
+                  ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                  ctypes.c_void_p]
+    return int(f(B, K, Hkv, d, cap, _DTYPE_CODE[k_cache.dtype], k_cache.data_ptr(), v_cache.data_ptr(),
+                 cache_len.data_ptr(), k_blk.data_ptr(), v_blk.data_ptr()))
+
+
+def commit_len(cache_len, n_commit, block: int, capacity: int) -> int:
+    """Step 2: cache_len += n_commit, in place.  Returns the C status."""
+    _check(cache_len, "cache_len")
+    _check(n_commit, "n_commit")
+    f = lib().oracle_commit_len
+    f.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
+    return int(f(cache_len.numel(), block, capacity, cache_len.data_ptr(), n_commit.data_ptr()))
+
+
+def rope_block(x: torch.Tensor, cache_len: torch.Tensor, theta: float = 10000.0) -> torch.Tensor:
+    """Rotary embedding of block tensor x [B][K][H][d] at positions cache_len[b] + i (half-split
+    pairing).  Returns float64 of the same shape."""
+    _check(x, "x")
+    _check(cache_len, "cache_len")
+    B, K, H, d = x.shape
+    y = torch.empty((B, K, H, d), dtype=torch.float64)
+    f = lib().oracle_rope_block
+    f.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                  ctypes.c_int32, ctypes.c_void_p, ctypes.c_double, ctypes.c_void_p]
+    rc = f(x.data_ptr(), _DTYPE_CODE[x.dtype], B, K, H, d, cache_len.data_ptr(), float(theta), y.data_ptr())
+    if rc != 0:
+        raise RuntimeError(f"oracle_rope_block failed ({rc})")
+    return y

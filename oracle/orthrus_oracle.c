@@ -25,7 +25,11 @@
  * the greedy rule at low temperature, library inverse-CDF on the degenerate
  * cases) and tests/test_oracle_lm_head_pins.py (planted maxima, exact-integer
  * logits against the logits-based rule, the library matrix product, ties, a
- * transposition trap).  Nothing is "parity unpinned".
+ * transposition trap), tests/test_oracle_truncate_rope_pins.py (the in-cache block
+ * against the library attention over one concatenated key sequence with an explicit
+ * mask; write + length bump against the append, byte for byte; the rotation against
+ * the transformers library's rotary embedding, its norm and relative-position
+ * properties) and tests/test_oracle_multiblock_pins.py.  Nothing is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -93,6 +97,9 @@ static int attend_row(const oracle_attn_t *a, int view, int b, int hq, int i,
     const int n_blk = (view == ORACLE_VIEW_DIFFUSION) ? K : i + 1;
     const int64_t n = P + n_blk;
     const double scale = a->scale > 0.0 ? a->scale : 1.0 / sqrt((double)d);
+    /* k_blk == NULL: the block's K/V rows are the cache rows [P_b, P_b + K) themselves
+     * (the pass wrote them there before attending; last paragraph of Section 3.3) */
+    const int in_cache = a->k_blk == NULL;
 
     double *s = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
     double *qv = (double *)malloc(sizeof(double) * (size_t)d);
@@ -111,10 +118,11 @@ static int attend_row(const oracle_attn_t *a, int view, int b, int hq, int i,
     }
     /* scores against the visible block rows */
     for (int ip = 0; ip < n_blk; ++ip) {
-        const int64_t off = (((int64_t)b * K + ip) * Hkv + h) * d;
+        const int64_t off = in_cache ? cache_base + (P + ip) * d : (((int64_t)b * K + ip) * Hkv + h) * d;
+        const void *src = in_cache ? a->k_cache : a->k_blk;
         double acc = 0.0;
         for (int c = 0; c < d; ++c)
-            acc += qv[c] * load_elem(a->k_blk, a->dtype, off + c);
+            acc += qv[c] * load_elem(src, a->dtype, off + c);
         s[P + ip] = acc * scale;
     }
 
@@ -131,9 +139,10 @@ static int attend_row(const oracle_attn_t *a, int view, int b, int hq, int i,
         for (int c = 0; c < d; ++c)
             out_row[c] += s[j] * load_elem(a->v_cache, a->dtype, cache_base + j * d + c);
     for (int ip = 0; ip < n_blk; ++ip) {
-        const int64_t off = (((int64_t)b * K + ip) * Hkv + h) * d;
+        const int64_t off = in_cache ? cache_base + (P + ip) * d : (((int64_t)b * K + ip) * Hkv + h) * d;
+        const void *src = in_cache ? a->v_cache : a->v_blk;
         for (int c = 0; c < d; ++c)
-            out_row[c] += s[P + ip] * load_elem(a->v_blk, a->dtype, off + c);
+            out_row[c] += s[P + ip] * load_elem(src, a->dtype, off + c);
     }
 
     if (w_row) {
@@ -451,6 +460,89 @@ int oracle_kv_append(int32_t B, int32_t K, int32_t Hkv, int32_t d, int64_t capac
         if (update_len) cache_len[b] = (int32_t)(P + n);
     }
     return rc;
+}
+
+/*
+ * Write-then-truncate form of the commit (last paragraph of Section 3.3: after the
+ * consensus the model "truncates the shared KV cache" to the accepted length).
+ *
+ * Step 1, oracle_block_kv_write: a pass writes the K/V rows of all K block positions
+ * behind the prefix, cache[b][h][P_b + i] = blk[b][i][h] for i < K, and leaves the
+ * length alone: rows at or beyond the length are dead, so the cache still denotes the
+ * same prefix.  The diffusion pass may park its transient block there, the AR pass
+ * overwrites it.  Returns -3 if a sequence has no room for K rows (it is skipped).
+ *
+ * Step 2, oracle_commit_len: the length grows by n_b; the rows beyond it, drafts the
+ * AR view did not confirm, are dead again.  Returns -3 for an n_b outside [0, K] or a
+ * length that would pass the capacity (that sequence keeps its length).
+ *
+ * Together, with the AR-view block written last, they leave rows [0, P_b + n_b) and
+ * the length exactly as oracle_kv_append does.
+ */
+int oracle_block_kv_write(int32_t B, int32_t K, int32_t Hkv, int32_t d, int64_t capacity,
+                          int dtype, void *k_cache, void *v_cache, const int32_t *cache_len,
+                          const void *k_blk, const void *v_blk)
+{
+    const size_t row = (size_t)d * elem_size(dtype);
+    int rc = 0;
+    for (int32_t b = 0; b < B; ++b) {
+        const int64_t P = cache_len[b];
+        if (P < 0 || P + K > capacity) { rc = -3; continue; }
+        for (int32_t i = 0; i < K; ++i)
+            for (int32_t h = 0; h < Hkv; ++h) {
+                const size_t src = ((((size_t)b * K + i) * Hkv) + h) * row;
+                const size_t dst = ((((size_t)b * Hkv + h) * (size_t)capacity) + (size_t)(P + i)) * row;
+                memcpy((char *)k_cache + dst, (const char *)k_blk + src, row);
+                memcpy((char *)v_cache + dst, (const char *)v_blk + src, row);
+            }
+    }
+    return rc;
+}
+
+int oracle_commit_len(int32_t B, int32_t K, int64_t capacity, int32_t *cache_len,
+                      const int32_t *n_commit)
+{
+    int rc = 0;
+    for (int32_t b = 0; b < B; ++b) {
+        const int64_t P = cache_len[b];
+        const int32_t n = n_commit[b];
+        if (n < 0 || n > K || P < 0 || P + n > capacity) { rc = -3; continue; }
+        cache_len[b] = (int32_t)(P + n);
+    }
+    return rc;
+}
+
+/*
+ * Rotary position embedding of a block, the step between the Q/K/V projections of a
+ * view (Section 3.1) and its attention: block row i of sequence b sits at position
+ * pos = P_b + i.  Head vectors are rotated pairwise in the half-split convention of
+ * the Qwen / Llama family the paper builds on (Section 4.1): for c < d/2,
+ *   angle = pos * theta^(-2c/d),
+ *   y[c]       = x[c] * cos(angle) - x[c + d/2] * sin(angle),
+ *   y[c + d/2] = x[c + d/2] * cos(angle) + x[c] * sin(angle).
+ * x: [B][K][H][d] of `dtype`; y: the same shape in double (the caller rounds).
+ */
+int oracle_rope_block(const void *x, int dtype, int32_t B, int32_t K, int32_t H, int32_t d,
+                      const int32_t *cache_len, double theta, double *y)
+{
+    if (d <= 0 || (d & 1) || theta <= 0.0) return -2;
+    const int half = d / 2;
+    for (int32_t b = 0; b < B; ++b)
+        for (int32_t i = 0; i < K; ++i) {
+            const double pos = (double)cache_len[b] + (double)i;
+            for (int32_t h = 0; h < H; ++h) {
+                const int64_t off = (((int64_t)b * K + i) * H + h) * d;
+                for (int c = 0; c < half; ++c) {
+                    const double ang = pos * pow(theta, -2.0 * (double)c / (double)d);
+                    const double cs = cos(ang), sn = sin(ang);
+                    const double x0 = load_elem(x, dtype, off + c);
+                    const double x1 = load_elem(x, dtype, off + c + half);
+                    y[off + c] = x0 * cs - x1 * sn;
+                    y[off + c + half] = x1 * cs + x0 * sn;
+                }
+            }
+        }
+    return 0;
 }
 
 int oracle_num_threads(void)
