@@ -16,7 +16,14 @@ import torch
 
 class Decoder:
     def __init__(self, binding, layers, hidden, n_q, n_kv, d, ffn, vocab, dtype, batch, capacity,
-                 block, seed=0, flags=0):
+                 block, seed=0, flags=0, commit_mode="append"):
+        """commit_mode "append": RoPE in torch, block K/V handed to the attention calls as tensors,
+        accepted rows copied by orthrus_kv_append_layers.  "truncate": the projection outputs go
+        through orthrus_rope_block_kv_write (rotation fused with the write of the block's K/V rows
+        behind the prefix), the attention calls read the block from the cache, and the commit is
+        orthrus_commit_len."""
+        assert commit_mode in ("append", "truncate")
+        self.commit_mode = commit_mode
         self.b, self.L, self.H, self.Hq, self.Hkv, self.d = binding, layers, hidden, n_q, n_kv, d
         self.V, self.dtype, self.B, self.cap, self.K = vocab, dtype, batch, capacity, block
         g = torch.Generator().manual_seed(seed)
@@ -70,11 +77,11 @@ class Decoder:
         x = self.norm(h)
         return h + (torch.nn.functional.silu(x @ lw["w1"]) * (x @ lw["w3"])) @ lw["w2"]
 
-    def layer_objs(self, block):
+    def layer_objs(self, block, extra_flags=0):
         b = self.b
         hint = self.cap - block
         return [b.make_layer(self.k_cache[l], self.v_cache[l], self.cache_len, self.Hq, block, hint, 0.0,
-                             self.flags) for l in range(self.L)]
+                             self.flags | extra_flags) for l in range(self.L)]
 
     # ------------------------------------------------------------------ prefill (torch)
     def prefill(self, prompt):
@@ -113,7 +120,8 @@ class Decoder:
         B = tokens.shape[0]
         h = self.emb[tokens.long()]
         pos = self.cache_len.long().unsqueeze(1) + torch.arange(block, device=h.device)
-        layers = self.layer_objs(block)
+        truncate = self.commit_mode == "truncate"
+        layers = self.layer_objs(block, b.LAYER_BLOCK_IN_CACHE if truncate else 0)
         # one workspace per block width, kept for good: captured graphs hold its address
         if block not in self._ws_by_block:
             self._ws_by_block[block] = b.new_workspace(b.orthrus_attend_workspace_bytes(layers[0]))
@@ -122,12 +130,22 @@ class Decoder:
         ks, vs = [], []
         for l, lw in enumerate(self.layers):
             x = self.norm(h)
-            q = self.rope((x @ lw["wq" + sfx]).view(B, block, self.Hq, self.d), pos).contiguous()
-            k = self.rope((x @ lw["wk" + sfx]).view(B, block, self.Hkv, self.d), pos).contiguous()
-            v = (x @ lw["wv" + sfx]).view(B, block, self.Hkv, self.d).contiguous()
-            out = torch.empty_like(q)
             fn = b.orthrus_diffusion_block_attend if view == "diff" else b.orthrus_ar_verify_attend
-            call = (lambda fn=fn, L=layers[l], q=q, k=k, v=v, out=out, ws=self.ws: fn(L, q, k, v, out, ws))
+            if truncate:
+                q_raw = (x @ lw["wq" + sfx]).view(B, block, self.Hq, self.d)
+                k = (x @ lw["wk" + sfx]).view(B, block, self.Hkv, self.d)
+                v = (x @ lw["wv" + sfx]).view(B, block, self.Hkv, self.d)
+                q = torch.empty_like(q_raw)
+                out = torch.empty_like(q)
+                call = (lambda fn=fn, L=layers[l], q_raw=q_raw, q=q, k=k, v=v, out=out, ws=self.ws:
+                        (b.orthrus_rope_block_kv_write(L, q_raw, k, v, 10000.0, q, ws),
+                         fn(L, q, None, None, out, ws)))
+            else:
+                q = self.rope((x @ lw["wq" + sfx]).view(B, block, self.Hq, self.d), pos).contiguous()
+                k = self.rope((x @ lw["wk" + sfx]).view(B, block, self.Hkv, self.d), pos).contiguous()
+                v = (x @ lw["wv" + sfx]).view(B, block, self.Hkv, self.d).contiguous()
+                out = torch.empty_like(q)
+                call = (lambda fn=fn, L=layers[l], q=q, k=k, v=v, out=out, ws=self.ws: fn(L, q, k, v, out, ws))
             call()
             if capture is not None and l in capture:
                 capture[l] = dict(q=q.clone(), k=k.clone(), v=v.clone(), out=out.clone(),
@@ -150,7 +168,11 @@ class Decoder:
         return self._lm_head_rows
 
     def commit(self, ks, vs, n_commit, block):
-        self.b.orthrus_kv_append_layers(self.layer_objs(block), ks, vs, n_commit, True, self.ws)
+        if self.commit_mode == "truncate":
+            # the AR pass left its block rows behind the prefix of every layer: only the length moves
+            self.b.orthrus_commit_len(self.layer_objs(block)[0], n_commit, self.ws)
+        else:
+            self.b.orthrus_kv_append_layers(self.layer_objs(block), ks, vs, n_commit, True, self.ws)
 
     def status(self):
         """OR of the device status words of every workspace this decoder has used."""

@@ -100,10 +100,19 @@ typedef struct {
  * is read early and any caller is safe.
  *
  * ORTHRUS_LAYER_NO_EARLY_LAUNCH: launch with ordinary stream order only.
+ *
+ * ORTHRUS_LAYER_BLOCK_IN_CACHE (attention calls only): the K/V rows of the block are not
+ * passed as tensors but already sit in the cache, at rows [P_b, P_b + K) of every KV
+ * head, where orthrus_block_kv_write or orthrus_rope_block_kv_write put them; the
+ * k_*_blk / v_*_blk arguments are ignored and may be NULL.  The masks are unchanged
+ * (diffusion view: all K rows; AR view: row i sees block rows 0..i).  Rows from P_b + K
+ * on are never read.  Compatible with ORTHRUS_LAYER_CACHE_QUIESCENT: the writing call
+ * touches only rows at or beyond cache_len.
  */
 enum {
     ORTHRUS_LAYER_CACHE_QUIESCENT = 1,
-    ORTHRUS_LAYER_NO_EARLY_LAUNCH = 2
+    ORTHRUS_LAYER_NO_EARLY_LAUNCH = 2,
+    ORTHRUS_LAYER_BLOCK_IN_CACHE = 4
 };
 
 /*
@@ -263,6 +272,43 @@ orthrus_status_t orthrus_lm_head_consensus(const void *hidden, const void *lm_he
 orthrus_status_t orthrus_kv_append(const orthrus_layer_t *layer, const void *k_ar_blk,
         const void *v_ar_blk, const int32_t *n_commit, int32_t update_len,
         void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The commit in its write-then-truncate form (last paragraph of Section 3.3: the model
+ * "truncates the shared KV cache" to the accepted length).  Instead of copying accepted
+ * rows after the consensus, every pass writes its whole block behind the prefix first:
+ *
+ * orthrus_block_kv_write: for every sequence b, KV head h and i < K,
+ *   k_cache[b][h][P_b + i] = k_blk[b][i][h]   (likewise v), a byte copy; cache_len is
+ *   not changed, so the rows are dead until a length says otherwise.  The diffusion pass
+ *   may park its transient block there; the AR pass of the same layer overwrites it.
+ *   A sequence with P_b + K > capacity is skipped (ORTHRUS_DEV_APPEND_OVERFLOW).
+ *
+ * orthrus_commit_len: cache_len[b] += n_commit[b] for the layer's length array (layers
+ * that share one array need one call).  An n_commit[b] outside [0, K] or a length that
+ * would pass the capacity leaves that length alone (ORTHRUS_DEV_APPEND_OVERFLOW).
+ * With the AR-view rows written last, rows [0, P_b + n) and the length end up exactly as
+ * orthrus_kv_append leaves them; the unconfirmed rows beyond are dead again.
+ *
+ * orthrus_rope_block_kv_write: the write fused with the rotary position embedding that
+ * sits between the projections (Section 3.1) and the attention.  Block row i of
+ * sequence b has position P_b + i; with the half-split pairing (c, c + d/2) and
+ *   angle = (P_b + i) * rope_theta^(-2c/d),
+ *   y[c] = x[c] cos(angle) - x[c + d/2] sin(angle),  y[c + d/2] = x[c + d/2] cos(angle) + x[c] sin(angle),
+ * q_out[b][i][hq] = rotate(q[b][i][hq]) (q_out may be q: in place), k_cache[b][h][P_b + i]
+ * = rotate(k_blk[b][i][h]), v_cache[b][h][P_b + i] = v_blk[b][i][h].  Angles are formed in
+ * double precision, results are rounded once to the layer's dtype.  q, q_out:
+ * [B][K][Hq][d]; k_blk, v_blk: [B][K][Hkv][d], straight from the projections (not rotated).
+ *
+ * `workspace` may be NULL in all three; if given, problems are reported through its status
+ * word.  One launch each.
+ */
+orthrus_status_t orthrus_block_kv_write(const orthrus_layer_t *layer, const void *k_blk, const void *v_blk,
+        void *workspace, size_t workspace_bytes, void *stream);
+orthrus_status_t orthrus_commit_len(const orthrus_layer_t *layer, const int32_t *n_commit,
+        void *workspace, size_t workspace_bytes, void *stream);
+orthrus_status_t orthrus_rope_block_kv_write(const orthrus_layer_t *layer, const void *q, const void *k_blk,
+        const void *v_blk, float rope_theta, void *q_out, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * The same commit for n_layers layers in one launch: the cycle's verify pass has

@@ -28,7 +28,8 @@ EXPORTS = [
     "orthrus_consensus_accept_static", "orthrus_consensus_sample_workspace_bytes",
     "orthrus_consensus_sample",
     "orthrus_lm_head_consensus_workspace_bytes", "orthrus_lm_head_consensus",
-    "orthrus_kv_append", "orthrus_kv_append_layers", "orthrus_read_status", "orthrus_set_path", "orthrus_last_path",
+    "orthrus_kv_append", "orthrus_kv_append_layers", "orthrus_block_kv_write", "orthrus_commit_len",
+    "orthrus_rope_block_kv_write", "orthrus_read_status", "orthrus_set_path", "orthrus_last_path",
     "orthrus_launch_count", "orthrus_status_string", "orthrus_version",
 ]
 
@@ -51,7 +52,7 @@ class Layer(ctypes.Structure):
                 ("flags", ctypes.c_uint32)]
 
 
-LAYER_CACHE_QUIESCENT, LAYER_NO_EARLY_LAUNCH = 1, 2
+LAYER_CACHE_QUIESCENT, LAYER_NO_EARLY_LAUNCH, LAYER_BLOCK_IN_CACHE = 1, 2, 4
 
 
 def _load() -> ctypes.CDLL:
@@ -90,6 +91,12 @@ def _load() -> ctypes.CDLL:
     lib.orthrus_kv_append_layers.restype = ctypes.c_int
     lib.orthrus_kv_append_layers.argtypes = [LP, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), vp, i32,
                                              vp, sz, vp]
+    lib.orthrus_block_kv_write.restype = ctypes.c_int
+    lib.orthrus_block_kv_write.argtypes = [LP, vp, vp, vp, sz, vp]
+    lib.orthrus_commit_len.restype = ctypes.c_int
+    lib.orthrus_commit_len.argtypes = [LP, vp, vp, sz, vp]
+    lib.orthrus_rope_block_kv_write.restype = ctypes.c_int
+    lib.orthrus_rope_block_kv_write.argtypes = [LP, vp, vp, vp, ctypes.c_float, vp, vp, sz, vp]
     lib.orthrus_read_status.restype = ctypes.c_int
     lib.orthrus_read_status.argtypes = [vp, vp, ctypes.POINTER(i32)]
     lib.orthrus_set_path.restype = ctypes.c_int
@@ -252,6 +259,31 @@ def orthrus_kv_append_layers(layers, k_ar_blks, v_ar_blks, n_commit, update_len:
     _check(_lib.orthrus_kv_append_layers(
         arr, n, kp, vp, _ptr(n_commit), 1 if update_len else 0, _ptr(workspace),
         0 if workspace is None else workspace.numel(), _stream(stream)), "orthrus_kv_append_layers")
+
+
+def _ws_args(workspace):
+    return _ptr(workspace), 0 if workspace is None else workspace.numel()
+
+
+def orthrus_block_kv_write(layer: Layer, k_blk, v_blk, workspace=None, stream=None) -> None:
+    """All K block rows go behind the prefix (cache rows [P_b, P_b + K)); lengths unchanged."""
+    _check(_lib.orthrus_block_kv_write(ctypes.byref(layer), _ptr(k_blk), _ptr(v_blk), *_ws_args(workspace),
+                                       _stream(stream)), "orthrus_block_kv_write")
+
+
+def orthrus_commit_len(layer: Layer, n_commit, workspace=None, stream=None) -> None:
+    """cache_len += n_commit for the layer's length array."""
+    _check(_lib.orthrus_commit_len(ctypes.byref(layer), _ptr(n_commit), *_ws_args(workspace), _stream(stream)),
+           "orthrus_commit_len")
+
+
+def orthrus_rope_block_kv_write(layer: Layer, q, k_blk, v_blk, rope_theta: float, q_out, workspace=None,
+                                stream=None) -> None:
+    """Rotary embedding of the block's queries (to q_out) and keys, keys and values written to
+    cache rows [P_b, P_b + K)."""
+    _check(_lib.orthrus_rope_block_kv_write(ctypes.byref(layer), _ptr(q), _ptr(k_blk), _ptr(v_blk),
+                                            float(rope_theta), _ptr(q_out), *_ws_args(workspace), _stream(stream)),
+           "orthrus_rope_block_kv_write")
 
 
 def orthrus_read_status(workspace, stream=None) -> int:

@@ -82,7 +82,8 @@ static orthrus_status_t check_layer(const orthrus_layer_t *L)
     if (L->block > L->capacity) return ORTHRUS_ERR_CAPACITY;
     if (L->capacity > 0x7fffffffLL) return ORTHRUS_ERR_UNSUPPORTED;
     if ((long long)L->max_len_hint + L->block > L->capacity) return ORTHRUS_ERR_CAPACITY;
-    if (L->flags & ~(uint32_t)(ORTHRUS_LAYER_CACHE_QUIESCENT | ORTHRUS_LAYER_NO_EARLY_LAUNCH))
+    if (L->flags & ~(uint32_t)(ORTHRUS_LAYER_CACHE_QUIESCENT | ORTHRUS_LAYER_NO_EARLY_LAUNCH |
+                               ORTHRUS_LAYER_BLOCK_IN_CACHE))
         return ORTHRUS_ERR_INVALID_ARG;
     return ORTHRUS_OK;
 }
@@ -183,7 +184,9 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
 {
     orthrus_status_t st = check_layer(L);
     if (st != ORTHRUS_OK) return st;
-    if (!q || !k_blk || !v_blk || !out || !ws || !L->k_cache || !L->v_cache || !L->cache_len)
+    const bool in_cache = (L->flags & ORTHRUS_LAYER_BLOCK_IN_CACHE) != 0;
+    if (in_cache) k_blk = v_blk = nullptr;    // not read in this mode
+    if (!q || (!in_cache && (!k_blk || !v_blk)) || !out || !ws || !L->k_cache || !L->v_cache || !L->cache_len)
         return ORTHRUS_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out) ||
         !aligned16(ws) || !aligned16(L->k_cache) || !aligned16(L->v_cache) ||
@@ -206,6 +209,7 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
     p.B = L->batch; p.K = L->block; p.Hq = L->n_q_heads; p.Hkv = L->n_kv_heads;
     p.G = p.Hq / p.Hkv; p.M = p.G * p.K; p.d = L->head_dim; p.capacity = L->capacity;
     p.chunk = pl.chunk; p.n_splits = pl.n_splits; p.causal = causal;
+    p.blk_in_cache = in_cache ? 1 : 0;
     const float scale = L->softmax_scale > 0.f ? L->softmax_scale : 1.f / sqrtf((float)p.d);
     p.scale_log2 = scale * 1.4426950408889634f;
 
@@ -415,6 +419,55 @@ orthrus_status_t orthrus_kv_append(const orthrus_layer_t *layer, const void *k_a
     cudaError_t e = launch_kv_append(*layer, k_ar_blk, v_ar_blk, n_commit, update_len,
                                      static_cast<int32_t *>(workspace),
                                      static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+}
+
+static orthrus_status_t check_block_call(const orthrus_layer_t *layer, void *workspace, size_t workspace_bytes)
+{
+    const orthrus_status_t st = check_layer(layer);
+    if (st != ORTHRUS_OK) return st;
+    if (!layer->k_cache || !layer->v_cache || !layer->cache_len) return ORTHRUS_ERR_INVALID_ARG;
+    if (!aligned16(layer->k_cache) || !aligned16(layer->v_cache) ||
+        (reinterpret_cast<uintptr_t>(layer->cache_len) & 3))
+        return ORTHRUS_ERR_INVALID_ARG;
+    if (workspace && (workspace_bytes < (size_t)kHeaderBytes || !aligned16(workspace)))
+        return ORTHRUS_ERR_WORKSPACE;
+    return ORTHRUS_OK;
+}
+
+orthrus_status_t orthrus_block_kv_write(const orthrus_layer_t *layer, const void *k_blk, const void *v_blk,
+        void *workspace, size_t workspace_bytes, void *stream)
+{
+    const orthrus_status_t st = check_block_call(layer, workspace, workspace_bytes);
+    if (st != ORTHRUS_OK) return st;
+    if (!k_blk || !v_blk || !aligned16(k_blk) || !aligned16(v_blk)) return ORTHRUS_ERR_INVALID_ARG;
+    cudaError_t e = launch_block_kv_write(*layer, k_blk, v_blk, static_cast<int32_t *>(workspace),
+                                          static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+}
+
+orthrus_status_t orthrus_commit_len(const orthrus_layer_t *layer, const int32_t *n_commit,
+        void *workspace, size_t workspace_bytes, void *stream)
+{
+    const orthrus_status_t st = check_block_call(layer, workspace, workspace_bytes);
+    if (st != ORTHRUS_OK) return st;
+    if (!n_commit || (reinterpret_cast<uintptr_t>(n_commit) & 3)) return ORTHRUS_ERR_INVALID_ARG;
+    cudaError_t e = launch_commit_len(*layer, n_commit, static_cast<int32_t *>(workspace),
+                                      static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+}
+
+orthrus_status_t orthrus_rope_block_kv_write(const orthrus_layer_t *layer, const void *q, const void *k_blk,
+        const void *v_blk, float rope_theta, void *q_out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    const orthrus_status_t st = check_block_call(layer, workspace, workspace_bytes);
+    if (st != ORTHRUS_OK) return st;
+    if (!q || !k_blk || !v_blk || !q_out || !aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) ||
+        !aligned16(q_out) || !(rope_theta > 0.f) || std::isinf(rope_theta))
+        return ORTHRUS_ERR_INVALID_ARG;
+    cudaError_t e = launch_rope_block_kv_write(*layer, q, k_blk, v_blk, (double)rope_theta, q_out,
+                                               static_cast<int32_t *>(workspace),
+                                               static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
 }
 

@@ -76,15 +76,18 @@ __global__ void __launch_bounds__(NWARPS * 32) attend_mma_kernel(AttnParams p)
 
     const __nv_bfloat16 *kc = static_cast<const __nv_bfloat16 *>(p.k_cache) + (long long)unit * p.capacity * HD;
     const __nv_bfloat16 *vc = static_cast<const __nv_bfloat16 *>(p.v_cache) + (long long)unit * p.capacity * HD;
-    const __nv_bfloat16 *kb = static_cast<const __nv_bfloat16 *>(p.k_blk) + ((long long)b * p.K * p.Hkv + h) * HD;
-    const __nv_bfloat16 *vb = static_cast<const __nv_bfloat16 *>(p.v_blk) + ((long long)b * p.K * p.Hkv + h) * HD;
+    // the block's rows: K rows of the block tensors, or the cache rows behind the prefix
+    const __nv_bfloat16 *kb = p.blk_in_cache ? kc + (long long)P * HD
+        : static_cast<const __nv_bfloat16 *>(p.k_blk) + ((long long)b * p.K * p.Hkv + h) * HD;
+    const __nv_bfloat16 *vb = p.blk_in_cache ? vc + (long long)P * HD
+        : static_cast<const __nv_bfloat16 *>(p.v_blk) + ((long long)b * p.K * p.Hkv + h) * HD;
 
     // tile t: block tile first (if this split owns it), then the prefix tiles
     auto issue_tile = [&](int t, int stage) {
         const bool is_blk = t < n_blk_tiles;
         const int base = is_blk ? 0 : pos0 + (t - n_blk_tiles) * TN;
         const int nv = is_blk ? p.K : min(TN, pos1 - base);
-        const long long row_stride = is_blk ? (long long)p.Hkv * HD : HD;
+        const long long row_stride = (is_blk && !p.blk_in_cache) ? (long long)p.Hkv * HD : HD;
         const __nv_bfloat16 *ks = is_blk ? kb : kc + (long long)base * HD;
         const __nv_bfloat16 *vs = is_blk ? vb : vc + (long long)base * HD;
         const uint32_t sk = smem_base + stage * 2 * TILE_BYTES;

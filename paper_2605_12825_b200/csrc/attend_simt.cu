@@ -73,7 +73,10 @@ __global__ void __launch_bounds__(128) attend_simt_kernel(AttnParams p)
             const int j = e / D, c = e % D;
             float kx = 0.f, vx = 0.f;
             if (j < nv) {
-                if (is_blk) {
+                if (is_blk && p.blk_in_cache) {
+                    const long long off = (long long)(P + base + j) * D + c;
+                    kx = to_f(kc[off]); vx = to_f(vc[off]);
+                } else if (is_blk) {
                     const long long off = (((long long)b * p.K + base + j) * p.Hkv + h) * D + c;
                     kx = to_f(kb[off]); vx = to_f(vb[off]);
                 } else {

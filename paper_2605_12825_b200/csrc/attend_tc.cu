@@ -233,6 +233,12 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             const int row = row_base + ((int)t0 + t) * TN;
             tma_load_2d(dst, m, 0, row, fb, stream_policy);
             tma_load_2d(dst + SUB_BYTES, m, 64, row, fb, stream_policy);
+        } else if (p.blk_in_cache) {
+            // block tile = the 64 cache rows from P on: rows >= K hold whatever follows the block
+            // (masked out of the scores; cleared in the V tile before its product)
+            const CUtensorMap *m = is_v ? &tm.v : &tm.k;
+            tma_load_2d(dst, m, 0, row_base + P, fb, stream_policy);
+            tma_load_2d(dst + SUB_BYTES, m, 64, row_base + P, fb, stream_policy);
         } else {                  // block tile: rows >= K are out of bounds and arrive as zeros
             const CUtensorMap *m = is_v ? &tm.vb : &tm.kb;
             tma_load_4d(dst, m, 0, h, 0, b, fb);
@@ -476,7 +482,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             if (!mbar_wait_warp(bar(BAR_FULL + slot), (j / NSLOT) & 1, abort_flag)) return false;
             // a ragged prefix tile: V rows past the prefix may hold anything, and 0 * NaN would
             // poison the product, so they are cleared before the MMA reads them
-            const int nv = t < n_mine ? min(TN, P - ((int)t0 + t) * TN) : TN;
+            const int nv = t < n_mine ? min(TN, P - ((int)t0 + t) * TN) : (p.blk_in_cache ? p.K : TN);
             if (nv < TN) {
                 unsigned char *vt = smem + OFF_RING + slot * SLOT_BYTES;
                 for (int e = lane; e < (TN - nv) * 16; e += 32) {
@@ -740,9 +746,13 @@ cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st)
     TcMaps tm;
     const unsigned long long rows = (unsigned long long)p.B * p.Hkv * p.capacity;
     if (!get_map(p.k_cache, rows, 0, 0, TN, 0, &tm.k) || !get_map(p.v_cache, rows, 0, 0, TN, 0, &tm.v) ||
-        !get_map(p.q, p.Hq, p.K, p.B, p.G, kb, &tm.q) ||
-        !get_map(p.k_blk, p.Hkv, p.K, p.B, 1, TN, &tm.kb) || !get_map(p.v_blk, p.Hkv, p.K, p.B, 1, TN, &tm.vb))
+        !get_map(p.q, p.Hq, p.K, p.B, p.G, kb, &tm.q))
         return cudaErrorInvalidValue;
+    if (p.blk_in_cache) {
+        tm.kb = tm.k; tm.vb = tm.v;           // unused: the block tile comes through the cache maps
+    } else if (!get_map(p.k_blk, p.Hkv, p.K, p.B, 1, TN, &tm.kb) || !get_map(p.v_blk, p.Hkv, p.K, p.B, 1, TN, &tm.vb)) {
+        return cudaErrorInvalidValue;
+    }
     return launch_tc(p, tm, kb, flags, st);
 }
 

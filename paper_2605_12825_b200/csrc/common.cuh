@@ -32,6 +32,7 @@ struct AttnParams {
     int chunk;          // prefix positions per split
     int n_splits;       // grid extent along the split axis
     int causal;         // 0: diffusion view (bidirectional block), 1: AR view (causal block)
+    int blk_in_cache;   // the block's K/V rows are the cache rows [P, P + K) (k_blk / v_blk unused)
     float scale_log2;   // softmax scale times log2(e)
 };
 
@@ -94,6 +95,13 @@ cudaError_t launch_consensus_static(const void *logits, int dtype, const int32_t
 cudaError_t launch_kv_append(const orthrus_layer_t &L, const void *k_blk, const void *v_blk,
                              const int32_t *n_commit, int update_len, int32_t *status,
                              cudaStream_t st);
+cudaError_t launch_block_kv_write(const orthrus_layer_t &L, const void *k_blk, const void *v_blk,
+                                  int32_t *status, cudaStream_t st);
+cudaError_t launch_commit_len(const orthrus_layer_t &L, const int32_t *n_commit, int32_t *status,
+                              cudaStream_t st);
+cudaError_t launch_rope_block_kv_write(const orthrus_layer_t &L, const void *q, const void *k_blk,
+                                       const void *v_blk, double theta, void *q_out, int32_t *status,
+                                       cudaStream_t st);
 
 size_t sample_workspace_bytes(int B, int K, int V);
 cudaError_t launch_consensus_sample(const void *ar_logits, const void *diff_logits, int dtype, const int32_t *draft,

@@ -61,7 +61,7 @@ def test_workspace_query_and_plan(lib):
 @pytest.mark.parametrize("bad,code", [
     (dict(n_q_heads=7), 1), (dict(head_dim=48), 2), (dict(block=65), 2), (dict(dtype=5), 2),
     (dict(max_len_hint=1020), 3), (dict(k_cache=0), 1), (dict(k_cache=0x1008), 1),
-    (dict(softmax_scale=-1.0), 1), (dict(flags=8), 1),
+    (dict(softmax_scale=-1.0), 1), (dict(flags=8), 1), (dict(flags=16), 1),
 ])
 def test_attend_rejects_bad_descriptors_before_launch(lib, bad, code):
     L = _layer(lib, **bad)
@@ -111,3 +111,26 @@ def test_lm_head_consensus_rejects_misuse_before_launch(lib):
     assert call(hidden=0x1008) == 1                # 16-byte alignment of the operands
     assert call(draft=0x3002) == 1
     assert call(wsb=1024) == 4
+
+
+def test_block_write_calls_reject_misuse_before_launch(lib):
+    L = _layer(lib)
+    n0 = lib.orthrus_launch_count()
+    w = lib.lib().orthrus_block_kv_write
+    assert w(ctypes.byref(L), None, 0x2000, None, 0, None) == 1
+    assert w(ctypes.byref(L), 0x1008, 0x2000, None, 0, None) == 1          # misaligned block tensor
+    assert w(ctypes.byref(L), 0x1000, 0x2000, 0x3000, 8, None) == 4        # workspace smaller than its header
+    assert w(None, 0x1000, 0x2000, None, 0, None) == 1
+    c = lib.lib().orthrus_commit_len
+    assert c(ctypes.byref(L), None, None, 0, None) == 1
+    assert c(ctypes.byref(L), 0x1002, None, 0, None) == 1
+    r = lib.lib().orthrus_rope_block_kv_write
+    assert r(ctypes.byref(L), 0x1000, 0x2000, 0x3000, 0.0, 0x4000, None, 0, None) == 1    # theta must be > 0
+    assert r(ctypes.byref(L), 0x1000, 0x2000, 0x3000, 1e4, None, None, 0, None) == 1
+    assert r(ctypes.byref(_layer(lib, head_dim=48)), 0x1000, 0x2000, 0x3000, 1e4, 0x4000, None, 0, None) == 2
+    # with the block in the cache the attention calls take no block tensors
+    A = _layer(lib, flags=4)
+    f = lib.lib().orthrus_ar_verify_attend
+    assert f(ctypes.byref(A), 0x4000, None, None, 0x7000, 0x8000, 16, None) == 4           # only the workspace is short
+    assert f(ctypes.byref(_layer(lib)), 0x4000, None, None, 0x7000, 0x8000, 1 << 30, None) == 1
+    assert lib.orthrus_launch_count() == n0
