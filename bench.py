@@ -702,6 +702,11 @@ def run_gpu(args):
         with torch.cuda.stream(stream):
             out["decoder_loop"] = decoder_loop_measure(B, dev, stream, 256 if cycles <= 0 else None,
                                                        cycles if cycles > 0 else None)
+            torch.cuda.empty_cache()
+            alt = decoder_loop_measure(B, dev, stream, 256 if cycles <= 0 else None,
+                                       cycles if cycles > 0 else None, commit_mode="truncate")
+            alt.pop("model"); alt.pop("lossless_check"); alt.pop("timed")
+            out["decoder_loop"]["truncate_commit"] = alt
     if rank == 0:
         print(json.dumps(out), flush=True)
     if dist is not None:
@@ -801,7 +806,7 @@ def lm_head_measure(B, wl, hidden_dim, dev, stream, steps, gpu_index=0):
             "roofline": roof}
 
 
-def decoder_loop_measure(B, dev, stream, n_new=256, max_cycles=None):
+def decoder_loop_measure(B, dev, stream, n_new=256, max_cycles=None, commit_mode="append"):
     """The end-to-end configuration: a random-initialised decoder (12 layers, hidden 2048, 16/4
     heads of 128, FFN 5632, vocabulary 32000, about 1.2 GB of bf16 weights per forward pass), 8
     prompts of 2048 tokens, then `n_new` generated tokens per sequence by repeated block-16
@@ -823,7 +828,7 @@ def decoder_loop_measure(B, dev, stream, n_new=256, max_cycles=None):
     g = torch.Generator().manual_seed(W.sub_seed(W.BASE_SEED, "cfg5_loop", 0, "prompt"))
     prompt = torch.randint(0, vocab, (Bt, T), generator=g).to(dev)
     dec = Decoder(B, layers, hidden, n_q, n_kv, d, ffn, vocab, torch.bfloat16, Bt, cap, K, seed=5,
-                  flags=B.LAYER_CACHE_QUIESCENT)
+                  flags=B.LAYER_CACHE_QUIESCENT, commit_mode=commit_mode)
     anchor0 = dec.prefill(prompt)
     loop = ForcedDraftLoop(dec, anchor0, rate, seed=W.sub_seed(W.BASE_SEED, "cfg5_loop", 0, "draft"), fused=True)
     len0 = dec.cache_len.clone()
@@ -889,7 +894,11 @@ def decoder_loop_measure(B, dev, stream, n_new=256, max_cycles=None):
     if status != 0:
         raise SystemExit(f"bench.py: device status word {status} after the decoder loop")
     ms = total_ms / cycles
-    return {"generated_tokens_per_sequence": n_new, "cycles": cycles, "ms_per_cycle": round(ms, 4),
+    return {"commit": "orthrus_kv_append_layers after the consensus; RoPE in torch" if commit_mode == "append" else
+                      "write-then-truncate: orthrus_rope_block_kv_write before every attention call (rotary "
+                      "embedding fused with the block write), attention reads the block from the cache, "
+                      "orthrus_commit_len after the consensus",
+            "generated_tokens_per_sequence": n_new, "cycles": cycles, "ms_per_cycle": round(ms, 4),
             "ms_per_cycle_median": round(statistics.median(cycle_ms), 4),
             "verified_tokens_per_s": round(tokens / (total_ms * 1e-3), 1),
             "verified_tokens": tokens,
