@@ -318,3 +318,31 @@ def rope_block(x: torch.Tensor, cache_len: torch.Tensor, theta: float = 10000.0)
     if rc != 0:
         raise RuntimeError(f"oracle_rope_block failed ({rc})")
     return y
+
+
+def multi_block_attend(q, k_blk, v_blk, k_cache, v_cache, cache_len, anchors,
+                       scale: Optional[float] = None) -> torch.Tensor:
+    """Diffusion-view attention under the multi-block mask of Eq. 6.  q [S][NB][K][Hq][d];
+    k_blk, v_blk [S][NB][K][Hkv][d]; cache [S][Hkv][capacity][d] holding cache_len[s] clean
+    positions; anchors int32 [S][NB].  Returns [S][NB][K][Hq][d] float64."""
+    S, NB, K, Hq, d = q.shape
+    Hkv = k_cache.shape[1]
+    for n_, t in (("q", q), ("k_blk", k_blk), ("v_blk", v_blk), ("k_cache", k_cache), ("v_cache", v_cache),
+                  ("cache_len", cache_len), ("anchors", anchors)):
+        _check(t, n_)
+    if tuple(k_blk.shape) != (S, NB, K, Hkv, d) or tuple(v_blk.shape) != (S, NB, K, Hkv, d):
+        raise ValueError("block KV must be [S][NB][K][Hkv][d]")
+    if anchors.dtype != torch.int32 or tuple(anchors.shape) != (S, NB):
+        raise ValueError("anchors must be int32 [S][NB]")
+    if int((anchors.long() > cache_len.long().view(S, 1)).sum()) or int((anchors < 0).sum()):
+        raise ValueError("anchors must lie in [0, cache_len]")
+    a = _AttnDesc(S, K, Hq, Hkv, d, _DTYPE_CODE[q.dtype], k_cache.shape[2], q.data_ptr(), k_blk.data_ptr(),
+                  v_blk.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), cache_len.data_ptr(),
+                  float(scale) if scale else 0.0)
+    out = torch.empty((S, NB, K, Hq, d), dtype=torch.float64)
+    f = lib().oracle_multi_block_attend
+    f.argtypes = [ctypes.POINTER(_AttnDesc), ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
+    rc = f(ctypes.byref(a), NB, anchors.data_ptr(), out.data_ptr())
+    if rc != 0:
+        raise RuntimeError(f"oracle_multi_block_attend failed ({rc})")
+    return out

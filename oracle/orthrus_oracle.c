@@ -202,6 +202,81 @@ int oracle_block_attend_rows(const oracle_attn_t *a, int view, const int32_t *ro
 }
 
 /*
+ * Multi-block diffusion-view attention, the training-time mask of Eq. 6 (Section 3.2).
+ *
+ * One clean sequence of L = cache_len[s] positions lives in the cache (the frozen AR
+ * view's K/V); NB blocks of K diffusion rows each are concatenated behind it, block j
+ * anchored at position a_j = anchors[s][j].  With q the row index among the NB*K
+ * diffusion rows and k the key index among the L + NB*K keys, Eq. 6 permits
+ *     k < L  and  k <= a_j - 1               (clean context before the block's anchor), or
+ *     k >= L and  floor(q / K) == floor((k - L) / K)   (the rows of the same block).
+ * The predicate is evaluated for every (q, k) exactly as printed; permitted keys enter
+ * one softmax with scale 1/sqrt(d).  q: [S][NB][K][Hq][d]; k_blk, v_blk: [S][NB][K][Hkv][d]
+ * (a->block = K, a->batch = S); out: [S][NB][K][Hq][d] doubles.
+ */
+int oracle_multi_block_attend(const oracle_attn_t *a, int32_t NB, const int32_t *anchors, double *out)
+{
+    const int S = a->batch, K = a->block, Hq = a->n_q_heads, Hkv = a->n_kv_heads, d = a->head_dim;
+    if (Hkv <= 0 || Hq % Hkv != 0 || NB <= 0) return -2;
+    const int G = Hq / Hkv;
+    const double scale = a->scale > 0.0 ? a->scale : 1.0 / sqrt((double)d);
+    int rc = 0;
+    const int64_t rows = (int64_t)S * NB * K * Hq;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < rows; ++r) {
+        const int hq = (int)(r % Hq);
+        const int64_t q = (r / Hq) % ((int64_t)NB * K);      /* row among the diffusion rows */
+        const int s = (int)(r / ((int64_t)Hq * NB * K));
+        const int h = hq / G;
+        const int64_t L = a->cache_len[s];
+        const int64_t n_keys = L + (int64_t)NB * K;
+        const int64_t anchor = anchors[(int64_t)s * NB + q / K];
+        double *w = (double *)malloc(sizeof(double) * (size_t)(n_keys > 0 ? n_keys : 1));
+        if (!w) {
+#pragma omp atomic write
+            rc = -1;
+            continue;
+        }
+        const int64_t q_off = r * d;
+        const int64_t cache_base = ((int64_t)s * Hkv + h) * a->capacity * d;
+        double mx = -INFINITY;
+        for (int64_t k = 0; k < n_keys; ++k) {
+            const int allowed = (k < L && k <= anchor - 1) || (k >= L && q / K == (k - L) / K);
+            if (!allowed) { w[k] = -INFINITY; continue; }
+            double acc = 0.0;
+            if (k < L) {
+                for (int c = 0; c < d; ++c)
+                    acc += load_elem(a->q, a->dtype, q_off + c) *
+                           load_elem(a->k_cache, a->dtype, cache_base + k * d + c);
+            } else {
+                const int64_t off = ((((int64_t)s * NB * K) + (k - L)) * Hkv + h) * d;
+                for (int c = 0; c < d; ++c)
+                    acc += load_elem(a->q, a->dtype, q_off + c) * load_elem(a->k_blk, a->dtype, off + c);
+            }
+            w[k] = acc * scale;
+            if (w[k] > mx) mx = w[k];
+        }
+        double den = 0.0;
+        for (int64_t k = 0; k < n_keys; ++k) { w[k] = exp(w[k] - mx); den += w[k]; }   /* exp(-inf) = 0 */
+        double *o = out + r * d;
+        for (int c = 0; c < d; ++c) o[c] = 0.0;
+        for (int64_t k = 0; k < n_keys; ++k) {
+            if (w[k] == 0.0) continue;
+            const double p = w[k] / den;
+            if (k < L) {
+                for (int c = 0; c < d; ++c)
+                    o[c] += p * load_elem(a->v_cache, a->dtype, cache_base + k * d + c);
+            } else {
+                const int64_t off = ((((int64_t)s * NB * K) + (k - L)) * Hkv + h) * d;
+                for (int c = 0; c < d; ++c) o[c] += p * load_elem(a->v_blk, a->dtype, off + c);
+            }
+        }
+        free(w);
+    }
+    return rc;
+}
+
+/*
  * Greedy consensus (Eq. 8 and the halt/commit rule of Section 3.3).
  *
  * Row i of the AR logits is conditioned on the anchor and drafts 0..i-1; its
