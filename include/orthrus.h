@@ -155,6 +155,28 @@ orthrus_status_t orthrus_ar_verify_attend(const orthrus_layer_t *layer,
         const void *q_ar, const void *k_ar_blk, const void *v_ar_blk, void *out,
         void *workspace, size_t workspace_bytes, void *stream);
 
+/*
+ * Diffusion-view attention under the multi-block mask of Eq. 6 (Section 3.2, the
+ * training-time form; inference is its single-block case): n_blocks blocks of K rows per
+ * sequence, block j of sequence s anchored at position anchors[s][j], all reading the one
+ * clean cache of their sequence.  Row i of block j attends to the cache rows
+ * [0, anchors[s][j]) of KV head hq/(Hq/Hkv) (rule (i): the clean context before its anchor)
+ * and to all K rows of its own block (rule (ii)), and to nothing else: not to other
+ * blocks, not to the context at or after its anchor.
+ *   q_diff, out            [S][n_blocks][K][Hq][d]
+ *   k_diff_blk, v_diff_blk [S][n_blocks][K][Hkv][d]
+ *   anchors                device int32 [S][n_blocks], 0 <= anchor <= capacity - K (values
+ *                          outside are clamped and flagged like a bad cache_len); the caller
+ *                          keeps them at or below the sequence's clean length
+ * layer describes the S sequences (batch = S; cache_len is not read; max_len_hint bounds
+ * the anchors).  Blocks are independent units of work, scheduled longest prefix first.
+ * Workspace: orthrus_multi_block_workspace_bytes(layer, n_blocks).
+ */
+size_t orthrus_multi_block_workspace_bytes(const orthrus_layer_t *layer, int32_t n_blocks);
+orthrus_status_t orthrus_multi_block_attend(const orthrus_layer_t *layer, int32_t n_blocks,
+        const int32_t *anchors, const void *q_diff, const void *k_diff_blk, const void *v_diff_blk,
+        void *out, void *workspace, size_t workspace_bytes, void *stream);
+
 /* Workspace bytes for orthrus_consensus_accept (header + per-row partial maxima). */
 size_t orthrus_consensus_workspace_bytes(int32_t batch, int32_t block, int32_t vocab);
 

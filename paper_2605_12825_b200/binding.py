@@ -24,6 +24,7 @@ DEV_BAD_CACHE_LEN, DEV_APPEND_OVERFLOW, DEV_WAIT_TIMEOUT = 1, 2, 4
 EXPORTS = [
     "orthrus_attend_workspace_bytes", "orthrus_workspace_init",
     "orthrus_diffusion_block_attend", "orthrus_ar_verify_attend",
+    "orthrus_multi_block_workspace_bytes", "orthrus_multi_block_attend",
     "orthrus_consensus_workspace_bytes", "orthrus_consensus_accept",
     "orthrus_consensus_accept_static", "orthrus_consensus_sample_workspace_bytes",
     "orthrus_consensus_sample",
@@ -71,6 +72,10 @@ def _load() -> ctypes.CDLL:
         f = getattr(lib, name)
         f.restype = ctypes.c_int
         f.argtypes = [LP, vp, vp, vp, vp, vp, sz, vp]
+    lib.orthrus_multi_block_workspace_bytes.restype = sz
+    lib.orthrus_multi_block_workspace_bytes.argtypes = [LP, i32]
+    lib.orthrus_multi_block_attend.restype = ctypes.c_int
+    lib.orthrus_multi_block_attend.argtypes = [LP, i32, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.orthrus_consensus_workspace_bytes.restype = sz
     lib.orthrus_consensus_workspace_bytes.argtypes = [i32, i32, i32]
     lib.orthrus_consensus_accept.restype = ctypes.c_int
@@ -176,6 +181,19 @@ def orthrus_ar_verify_attend(layer: Layer, q_ar, k_ar_blk, v_ar_blk, out, worksp
     _check(_lib.orthrus_ar_verify_attend(
         ctypes.byref(layer), _ptr(q_ar), _ptr(k_ar_blk), _ptr(v_ar_blk), _ptr(out),
         _ptr(workspace), workspace.numel(), _stream(stream)), "orthrus_ar_verify_attend")
+
+
+def orthrus_multi_block_workspace_bytes(layer: Layer, n_blocks: int) -> int:
+    return int(_lib.orthrus_multi_block_workspace_bytes(ctypes.byref(layer), n_blocks))
+
+
+def orthrus_multi_block_attend(layer: Layer, anchors, q_diff, k_diff_blk, v_diff_blk, out, workspace,
+                               stream=None) -> None:
+    """Diffusion-view attention under the multi-block mask of Eq. 6; anchors int32 [S][n_blocks],
+    q_diff / out [S][n_blocks][K][Hq][d], block K/V [S][n_blocks][K][Hkv][d]."""
+    _check(_lib.orthrus_multi_block_attend(
+        ctypes.byref(layer), anchors.shape[1], _ptr(anchors), _ptr(q_diff), _ptr(k_diff_blk), _ptr(v_diff_blk),
+        _ptr(out), _ptr(workspace), workspace.numel(), _stream(stream)), "orthrus_multi_block_attend")
 
 
 def orthrus_consensus_workspace_bytes(batch: int, block: int, vocab: int) -> int:

@@ -178,9 +178,11 @@ static size_t partial_bytes(const orthrus_layer_t *L, const Plan &pl, size_t *ml
     return o_bytes + ml_bytes;
 }
 
+// nb: blocks per sequence (the batch of *L then counts blocks, and batch entry b reads the cache
+// of sequence b / nb)
 static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void *q,
                                const void *k_blk, const void *v_blk, void *out, void *ws,
-                               size_t ws_bytes, void *stream)
+                               size_t ws_bytes, void *stream, int nb = 1)
 {
     orthrus_status_t st = check_layer(L);
     if (st != ORTHRUS_OK) return st;
@@ -210,6 +212,7 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
     p.G = p.Hq / p.Hkv; p.M = p.G * p.K; p.d = L->head_dim; p.capacity = L->capacity;
     p.chunk = pl.chunk; p.n_splits = pl.n_splits; p.causal = causal;
     p.blk_in_cache = in_cache ? 1 : 0;
+    p.nb = nb; p.len_cap = L->capacity - L->block;
     const float scale = L->softmax_scale > 0.f ? L->softmax_scale : 1.f / sqrtf((float)p.d);
     p.scale_log2 = scale * 1.4426950408889634f;
 
@@ -274,6 +277,36 @@ orthrus_status_t orthrus_ar_verify_attend(const orthrus_layer_t *layer, const vo
         size_t workspace_bytes, void *stream)
 {
     return attend(layer, 1, q_ar, k_ar_blk, v_ar_blk, out, workspace, workspace_bytes, stream);
+}
+
+// Eq. 6 as a batch of blocks: the descriptor of S sequences becomes one of S * n_blocks batch
+// entries whose prefix lengths are the anchors; entry b reads the cache of sequence b / n_blocks.
+static bool multi_block_layer(const orthrus_layer_t *layer, int32_t n_blocks, const int32_t *anchors,
+                              orthrus_layer_t *out)
+{
+    if (!layer || n_blocks < 1 || layer->batch < 1 || (long long)layer->batch * n_blocks > 0x7fffffffLL) return false;
+    *out = *layer;
+    out->batch = layer->batch * n_blocks;
+    out->cache_len = const_cast<int32_t *>(anchors);
+    out->flags = layer->flags & ~(uint32_t)ORTHRUS_LAYER_BLOCK_IN_CACHE;
+    return true;
+}
+
+size_t orthrus_multi_block_workspace_bytes(const orthrus_layer_t *layer, int32_t n_blocks)
+{
+    orthrus_layer_t L;
+    if (!multi_block_layer(layer, n_blocks, nullptr, &L)) return 0;
+    return orthrus_attend_workspace_bytes(&L);
+}
+
+orthrus_status_t orthrus_multi_block_attend(const orthrus_layer_t *layer, int32_t n_blocks,
+        const int32_t *anchors, const void *q_diff, const void *k_diff_blk, const void *v_diff_blk,
+        void *out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    orthrus_layer_t L;
+    if (!anchors || !multi_block_layer(layer, n_blocks, anchors, &L)) return ORTHRUS_ERR_INVALID_ARG;
+    if (layer->flags & ORTHRUS_LAYER_BLOCK_IN_CACHE) return ORTHRUS_ERR_INVALID_ARG;
+    return attend(&L, 0, q_diff, k_diff_blk, v_diff_blk, out, workspace, workspace_bytes, stream, n_blocks);
 }
 
 size_t orthrus_consensus_workspace_bytes(int32_t batch, int32_t block, int32_t vocab)

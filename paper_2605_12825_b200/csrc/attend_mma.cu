@@ -74,8 +74,9 @@ __global__ void __launch_bounds__(NWARPS * 32) attend_mma_kernel(AttnParams p)
     const int gq = lane >> 2, tq = lane & 3;               // row within 8, column pair
     const uint32_t smem_base = smem_u32(smem_raw);
 
-    const __nv_bfloat16 *kc = static_cast<const __nv_bfloat16 *>(p.k_cache) + (long long)unit * p.capacity * HD;
-    const __nv_bfloat16 *vc = static_cast<const __nv_bfloat16 *>(p.v_cache) + (long long)unit * p.capacity * HD;
+    const long long cache_unit = (long long)(b / p.nb) * p.Hkv + h;      // whose cache this batch entry reads
+    const __nv_bfloat16 *kc = static_cast<const __nv_bfloat16 *>(p.k_cache) + cache_unit * p.capacity * HD;
+    const __nv_bfloat16 *vc = static_cast<const __nv_bfloat16 *>(p.v_cache) + cache_unit * p.capacity * HD;
     // the block's rows: K rows of the block tensors, or the cache rows behind the prefix
     const __nv_bfloat16 *kb = p.blk_in_cache ? kc + (long long)P * HD
         : static_cast<const __nv_bfloat16 *>(p.k_blk) + ((long long)b * p.K * p.Hkv + h) * HD;

@@ -39,8 +39,9 @@ __global__ void __launch_bounds__(128) attend_simt_kernel(AttnParams p)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const T *q = static_cast<const T *>(p.q);
-    const T *kc = static_cast<const T *>(p.k_cache) + ((long long)unit * p.capacity) * D;
-    const T *vc = static_cast<const T *>(p.v_cache) + ((long long)unit * p.capacity) * D;
+    const long long cache_unit = (long long)(b / p.nb) * p.Hkv + h;      // whose cache this batch entry reads
+    const T *kc = static_cast<const T *>(p.k_cache) + (cache_unit * p.capacity) * D;
+    const T *vc = static_cast<const T *>(p.v_cache) + (cache_unit * p.capacity) * D;
     const T *kb = static_cast<const T *>(p.k_blk);
     const T *vb = static_cast<const T *>(p.v_blk);
 

@@ -184,7 +184,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     // clusters are ordered longest prefix first (ties by sequence index)
     int b = order / p.Hkv;
     const int h = order % p.Hkv;
-    const int len_hi = (int)(p.capacity - p.K);
+    const int len_hi = (int)p.len_cap;
     if (p.B > 1 && p.B <= 128) {
         const int want = b;
         for (int i = tid; i < p.B; i += NTHREADS) {
@@ -212,7 +212,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     const bool owner = rank == S - 1;                         // its last tile is the block tile
     const int n_mine = n_tiles - (owner ? 1 : 0);             // prefix tiles of this CTA
     const bool active = n_tiles > 0 && aligned;
-    const int row_base = (int)(((long long)b * p.Hkv + h) * p.capacity);   // row of position 0
+    const int row_base = (int)(((long long)(b / p.nb) * p.Hkv + h) * p.capacity);   // row of position 0
 
     // The ring holds K and V tiles in the order the MMAs consume them: K0, K1, V0, K2, V1, ...,
     // K(n-1), V(n-2), V(n-1) (the product P.V of a tile is issued after the scores of the next
@@ -744,7 +744,7 @@ cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st)
 {
     const int kb = tc_kb_rows(p.G, p.K);
     TcMaps tm;
-    const unsigned long long rows = (unsigned long long)p.B * p.Hkv * p.capacity;
+    const unsigned long long rows = (unsigned long long)(p.B / p.nb) * p.Hkv * p.capacity;
     if (!get_map(p.k_cache, rows, 0, 0, TN, 0, &tm.k) || !get_map(p.v_cache, rows, 0, 0, TN, 0, &tm.v) ||
         !get_map(p.q, p.Hq, p.K, p.B, p.G, kb, &tm.q))
         return cudaErrorInvalidValue;

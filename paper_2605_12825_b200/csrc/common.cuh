@@ -33,6 +33,10 @@ struct AttnParams {
     int n_splits;       // grid extent along the split axis
     int causal;         // 0: diffusion view (bidirectional block), 1: AR view (causal block)
     int blk_in_cache;   // the block's K/V rows are the cache rows [P, P + K) (k_blk / v_blk unused)
+    int nb;             // blocks per sequence: batch entry b reads the cache of sequence b / nb
+                        // (1 except for the multi-block mask of Eq. 6, where B counts blocks)
+    long long len_cap;  // largest admissible prefix length (capacity - K; capacity for Eq. 6,
+                        // whose blocks are never stored behind their prefix)
     float scale_log2;   // softmax scale times log2(e)
 };
 
@@ -46,7 +50,7 @@ __host__ __device__ inline int last_split(int P, int chunk) {
 // Largest prefix length a launch can serve: the capacity left beside the block, and (split-KV
 // grids of the SIMT / mma paths, sized from max_len_hint) what the planned splits cover.
 __host__ __device__ inline long long max_served_len(const AttnParams &p) {
-    const long long hi = p.capacity - p.K;
+    const long long hi = p.len_cap;
     const long long planned = (long long)p.n_splits * p.chunk;
     return planned < hi ? planned : hi;
 }
