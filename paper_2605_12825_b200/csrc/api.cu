@@ -122,8 +122,9 @@ static Plan make_plan(const orthrus_layer_t *L, bool tc)
         // as many splits as still fit on the GPU in one wave.  Many units: just enough CTAs
         // to fill every slot once; sequences of unequal length are handed out longest first.
         const int tn = tc_tile_positions();
-        const int units = L->batch * L->n_kv_heads * tc_row_tiles(L->n_q_heads / L->n_kv_heads, L->block);
-        const int slots = tc_ctas_per_sm() * num_sms();
+        const int G = L->n_q_heads / L->n_kv_heads, nt = tc_tiles_per_cta(G, L->block);
+        const int units = L->batch * L->n_kv_heads * tc_cta_groups(G, L->block);
+        const int slots = tc_ctas_per_sm(nt) * num_sms();
         const int tiles = max_len > 0 ? (max_len + tn - 1) / tn : 1;
         int S = 1;
         if (forced > 0) {
@@ -136,7 +137,7 @@ static Plan make_plan(const orthrus_layer_t *L, bool tc)
             //  still split; many small CTAs would spend their time starting and merging)
             while (S < 16 && units * S < slots && tiles / (S * 2) >= 8) S *= 2;
         }
-        const int max_cluster = tc_max_cluster();
+        const int max_cluster = tc_max_cluster(nt);
         if (S > max_cluster) S = max_cluster;
         if (S > tiles) S = tiles;
         if (S < 1) S = 1;

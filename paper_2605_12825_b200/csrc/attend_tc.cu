@@ -58,39 +58,59 @@ namespace {
 constexpr int HD = 128;                  // head_dim
 constexpr int MROWS = 128;               // MMA M
 constexpr int TN = 64;                   // key positions per tile
-constexpr int NTHREADS = 192;
-constexpr int NSLOT = 5;                 // ring slots, one K or V tile each
 constexpr int QSUB_BYTES = MROWS * 128;  // a [128 rows][64 cols] bf16 sub-tile of Q
 constexpr int SUB_BYTES = TN * 128;      // a [64 rows][64 cols] bf16 sub-tile of K or V
 constexpr int SLOT_BYTES = 2 * SUB_BYTES;
+constexpr int MAX_BARS = 40;
 
-// shared memory map (offsets from a 1024-byte aligned base)
-constexpr int OFF_Q = 0;                                   // [128][128] bf16, 2 sub-tiles
-constexpr int OFF_RING = OFF_Q + 2 * QSUB_BYTES;           // NSLOT x 16 KB
-constexpr int OFF_BAR = OFF_RING + NSLOT * SLOT_BYTES;     // mbarriers
-constexpr int OFF_MISC = OFF_BAR + 24 * 8;                 // tmem base, abort flag, unit
-constexpr int SMEM_BYTES = OFF_MISC + 64;
-static_assert(2 * (SMEM_BYTES + 1024) <= 228 * 1024, "two CTAs per SM");
-
-enum { BAR_FULL = 0, BAR_EMPTY = NSLOT, BAR_QFULL = 2 * NSLOT, BAR_SFULL, BAR_PFULL = BAR_SFULL + 2,
-       BAR_PVDONE = BAR_PFULL + 2, BAR_ALLDONE, NUM_BARS };
-static_assert(NUM_BARS <= 24, "barrier area");
-
-constexpr uint32_t TM_O = 0, TM_S = 128, TM_COLS = 256;   // TMEM column map
+// Two shapes of CTA.  NT = 1: one 128-row query tile, 192 threads, 112 KB of shared memory and
+// 256 TMEM columns, so that two CTAs share an SM.  NT = 2 (units wider than 128 rows): two
+// 128-row query tiles of the same unit share ONE ring of K/V tiles, so every cache byte is
+// loaded once for both; 320 threads (two softmax warpgroups), 224 KB of shared memory, all
+// 512 TMEM columns: one CTA per SM, with a ring twice as deep.
+template <int NT> struct Shape {
+    static constexpr int NSLOT = NT == 1 ? 5 : 10;             // ring slots, one K or V tile each
+    // warps: 4 softmax warps per query tile, the producer, one MMA-issuing warp per query tile
+    // (a thread is held for about a hundred cycles per tcgen05.mma it issues, whatever the
+    //  shape: the two tiles' MMAs of a key tile are issued side by side, not one after the other)
+    static constexpr int NTHREADS = 32 * (4 * NT + 1 + NT);
+    static constexpr int PRODUCER_WARP = 4 * NT, MMA_WARP = 4 * NT + 1;    // MMA warps: MMA_WARP + ti
+    // shared memory map (offsets from a 1024-byte aligned base)
+    static constexpr int OFF_Q = 0;                            // NT x [128][128] bf16, 2 sub-tiles each
+    static constexpr int OFF_RING = OFF_Q + NT * 2 * QSUB_BYTES;
+    static constexpr int OFF_BAR = OFF_RING + NSLOT * SLOT_BYTES;
+    static constexpr int OFF_MISC = OFF_BAR + MAX_BARS * 8;    // tmem base, abort flag, unit
+    static constexpr int SMEM_BYTES = OFF_MISC + 64;
+    // mbarriers: per ring slot, per query tile and score buffer
+    static constexpr int BAR_FULL = 0, BAR_EMPTY = NSLOT, BAR_QFULL = 2 * NSLOT;
+    static constexpr int BAR_SFULL = BAR_QFULL + 1;            // + ti * 2 + buffer
+    static constexpr int BAR_PFULL = BAR_SFULL + 2 * NT;       // + ti * 2 + buffer
+    static constexpr int BAR_PVDONE = BAR_PFULL + 2 * NT;      // + ti
+    static constexpr int BAR_ALLDONE = BAR_PVDONE + NT;        // + ti
+    static constexpr int NUM_BARS = BAR_ALLDONE + NT;
+    static_assert(NUM_BARS <= MAX_BARS, "barrier area");
+    // TMEM columns: the NT output accumulators, then two score buffers per query tile
+    static constexpr uint32_t TM_COLS = 256 * NT;
+    static constexpr uint32_t tm_o(int ti) { return (uint32_t)ti * HD; }
+    static constexpr uint32_t tm_s(int ti, int sb) { return (uint32_t)(NT * HD + ti * 2 * TN + sb * TN); }
+};
+static_assert(2 * (Shape<1>::SMEM_BYTES + 1024) <= 228 * 1024, "two CTAs per SM");
+static_assert(Shape<2>::SMEM_BYTES <= 227 * 1024, "one CTA per SM");
 constexpr float RESCALE_THRESHOLD = 8.f;                  // log2 units
 struct TcMaps { CUtensorMap k, v, q, kb, vb; };
 
 // Merge through the workspace.  A task is (32-row group, 16-byte column chunk) of a unit; lane =
 // row of the group.  Tasks go round-robin to the cluster's CTAs and their warps.  A warp takes
-// 16 / SP tasks per round (SP = cluster size rounded up to a power of two), so that sixteen
-// 16-byte loads per lane are in flight whatever the cluster size; every load of a warp covers
+// LOADS / SP tasks per round (SP = cluster size rounded up to a power of two), so that LOADS
+// 16-byte loads per lane are in flight whatever the cluster size (sixteen in the narrow shape,
+// eight in the wide one, which has fewer registers per thread); every load of a warp covers
 // 512 contiguous bytes.  grp_o: the cluster's S partial tiles, each [32 chunks][128 rows] of
 // float4; grp_ml: (max, sum) per [CTA][row].  store(R, chunk, acc, 1 / sum).
-template <int SP, class Store>
+template <int SP, int LOADS, class Store>
 __device__ inline void l2_merge_tasks(int S, int rank, int warp, int lane, int n_warps, int n_tasks, int rows_here,
                                       const float4 *grp_o, const float2 *grp_ml, Store store)
 {
-    constexpr int TB = 16 / SP;
+    constexpr int TB = LOADS / SP > 0 ? LOADS / SP : 1;
     // task index of (round, slot u) for this warp: consecutive tasks of a round sit S * n_warps apart
     for (int t0 = rank + warp * S; t0 < n_tasks; t0 += S * n_warps * TB) {
         float2 ml[TB][SP];
@@ -132,12 +152,41 @@ __device__ inline void l2_merge_tasks(int S, int rank, int warp, int lane, int n
     }
 }
 
-// Thread r of the softmax warps owns query row r (TMEM lane r) and all 64 columns of a tile.
-__global__ void __launch_bounds__(NTHREADS, 2)
+// One query tile's merge, kept out of line so that its registers (sixteen 16-byte loads in flight
+// per lane) do not add to those of the streaming loop.  out_tile: the output row of the tile's
+// first block position and first head of the group; row R = i * G + g lies (i * Hq + g) rows on.
+template <int LOADS>
+__device__ __noinline__ void merge_tile(int S, int rank, int warp, int lane, int n_warps, int rows_here,
+                                        const float4 *grp_o, const float2 *grp_ml, __nv_bfloat16 *out_tile,
+                                        int G, int Hq)
+{
+    const int n_tasks = ((rows_here + 31) >> 5) * (HD / 4);
+    auto run = [&](auto sp) {
+        l2_merge_tasks<decltype(sp)::value, LOADS>(S, rank, warp, lane, n_warps, n_tasks, rows_here, grp_o, grp_ml,
+                                            [&](int R, int c, const float4 &acc, float inv) {
+            __nv_bfloat16 *row = out_tile + ((long long)(R / G) * Hq + R % G) * HD;
+            reinterpret_cast<uint2 *>(row)[c] =
+                make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+        });
+    };
+    if (S <= 2) run(std::integral_constant<int, 2>());
+    else if (S <= 4) run(std::integral_constant<int, 4>());
+    else if (S <= 8) run(std::integral_constant<int, 8>());
+    else run(std::integral_constant<int, 16>());
+}
+
+// Thread r of a softmax warpgroup owns query row r of its tile (TMEM lane r) and all 64 columns of
+// a key tile.  blockIdx.z counts groups of NT query tiles; warpgroup ti works on tile z * NT + ti.
+template <int NT>
+__global__ void __launch_bounds__(Shape<NT>::NTHREADS, NT == 1 ? 2 : 1)
 attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const int S, const int kb_rows,
                  const int quiescent)
 {
+    using C = Shape<NT>;
     constexpr int W = TN;                     // score columns per softmax thread
+    constexpr int NSLOT = C::NSLOT, NTHREADS = C::NTHREADS;
+    constexpr int OFF_Q = C::OFF_Q, OFF_RING = C::OFF_RING, OFF_BAR = C::OFF_BAR, OFF_MISC = C::OFF_MISC;
+    constexpr int BAR_FULL = C::BAR_FULL, BAR_EMPTY = C::BAR_EMPTY, BAR_QFULL = C::BAR_QFULL;
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t sbase = smem_u32(smem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + OFF_MISC + 8);
@@ -147,29 +196,39 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int rank = S > 1 ? (int)cluster_rank() : 0;
-    const int order = blockIdx.y, rt = blockIdx.z;
-    // this row tile: kb_rows block positions x G heads (at most 128 rows)
-    const int i0 = rt * kb_rows;
-    const int rows_here = min(p.K - i0, kb_rows) * p.G;
-    const int n_act = (rows_here + 31) >> 5;                  // softmax warps with rows
+    const int order = blockIdx.y;
+    // query tile ti of this CTA: kb_rows block positions x G heads (at most 128 rows); the last
+    // group of a unit may hold fewer than NT tiles
+    auto tile_i0 = [&](int ti) { return ((int)blockIdx.z * NT + ti) * kb_rows; };
+    auto tile_rows = [&](int ti) { return max(0, min(p.K - tile_i0(ti), kb_rows)) * p.G; };
     const bool aligned = (sbase & 1023u) == 0;                // swizzled tiles need 1 KB alignment
 
     // ------------------------------------------------------------------ prologue
     if (tid == 0) { *abort_flag = aligned ? 0 : 1; *seq_slot = 0; }
-    if (warp == 4 && lane == 0) {
-        for (int i = 0; i < 2 * NSLOT; ++i) mbar_init(bar(i), 1);
+    if (warp == C::PRODUCER_WARP && lane == 0) {
+        int n_tiles_q = 0;                                    // query tiles with rows = MMA warps at work
+        for (int ti = 0; ti < NT; ++ti) n_tiles_q += tile_rows(ti) > 0;
+        for (int i = 0; i < NSLOT; ++i) {
+            mbar_init(bar(BAR_FULL + i), 1);
+            mbar_init(bar(BAR_EMPTY + i), max(1, n_tiles_q));  // every MMA warp releases a slot
+        }
         mbar_init(bar(BAR_QFULL), 1);
-        mbar_init(bar(BAR_SFULL), 1); mbar_init(bar(BAR_SFULL + 1), 1);
-        mbar_init(bar(BAR_PFULL), n_act); mbar_init(bar(BAR_PFULL + 1), n_act);
-        mbar_init(bar(BAR_PVDONE), 1);
-        mbar_init(bar(BAR_ALLDONE), 1);
+        for (int ti = 0; ti < NT; ++ti) {
+            const int n_act = max(1, (tile_rows(ti) + 31) >> 5);      // softmax warps with rows
+            for (int sb = 0; sb < 2; ++sb) {
+                mbar_init(bar(C::BAR_SFULL + ti * 2 + sb), 1);
+                mbar_init(bar(C::BAR_PFULL + ti * 2 + sb), n_act);
+            }
+            mbar_init(bar(C::BAR_PVDONE + ti), 1);
+            mbar_init(bar(C::BAR_ALLDONE + ti), 1);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
         prefetch_map(&tm.k); prefetch_map(&tm.v); prefetch_map(&tm.q);
         prefetch_map(&tm.kb); prefetch_map(&tm.vb);
-    } else if (warp == 5) {
+    } else if (warp == C::MMA_WARP) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"(TM_COLS) : "memory");
+                     ::"r"(smem_u32(tmem_slot)), "r"(C::TM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -249,7 +308,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     if (quiescent) {
         // the cache rows below cache_len are not being written by the preceding kernel:
         // request the first prefix tiles before waiting for it
-        if (active && warp == 4 && lane == 0)
+        if (active && warp == C::PRODUCER_WARP && lane == 0)
             while (produced < (owner ? item_of_k(n_tiles - 1) : 2 * n_tiles) && produced < NSLOT) {
                 issue_item(produced); ++produced;     // (stops before the block tile's first item)
             }
@@ -257,12 +316,15 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     }
     griddep_launch();
 
-    if (warp < 4) {
-        const int r = tid;
+    if (warp < 4 * NT) {
+        const int ti = warp >> 2, wq = warp & 3;              // query tile, quarter of its TMEM lanes
+        const int r = tid - ti * MROWS;
+        const int rows_here = tile_rows(ti);
         const bool valid = r < rows_here;
-        const bool warp_active = warp * 32 < rows_here;
-        const int i_row = i0 + r / p.G;
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        const bool warp_active = wq * 32 < rows_here;
+        const int i_row = tile_i0(ti) + r / p.G;
+        const uint32_t lane_base = tmem + ((uint32_t)(wq * 32) << 16);
+        const uint32_t TM_O = C::tm_o(ti);
         float m_run = -INFINITY, l_run = 0.f;
         bool have_o = false;
         if (active && warp_active) {
@@ -272,12 +334,13 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             bool ok = true;
             for (int t = 0; t < n_tiles; ++t) {
                 const int sb = t & 1;
-                ok = mbar_wait_warp(bar(BAR_SFULL + sb), (t >> 1) & 1, abort_flag);
+                ok = mbar_wait_warp(bar(C::BAR_SFULL + ti * 2 + sb), (t >> 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
+                const uint32_t TM_S = C::tm_s(ti, sb);
                 uint32_t s[W];
 #pragma unroll
-                for (int c = 0; c < W / 32; ++c) tmem_ld32(lane_base + TM_S + sb * TN + c * 32, s + c * 32);
+                for (int c = 0; c < W / 32; ++c) tmem_ld32(lane_base + TM_S + c * 32, s + c * 32);
                 tmem_ld_wait();
                 // visible columns of this row in this tile
                 int lim;
@@ -316,7 +379,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                     if (need) { m_run = m_new; l_run *= alpha; }
                     if (t > 0) {
                         // O holds the products of tiles 0..t-1 and nothing is adding to it now
-                        ok = mbar_wait_warp(bar(BAR_PVDONE), (t - 1) & 1, abort_flag);
+                        ok = mbar_wait_warp(bar(C::BAR_PVDONE + ti), (t - 1) & 1, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
 #pragma unroll 1
@@ -366,15 +429,15 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                 }
                 l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
                 // P over the scores, 2 bf16 per 32-bit column
-                tmem_st32(lane_base + TM_S + sb * TN, pk);
+                tmem_st32(lane_base + TM_S, pk);
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_PFULL + sb));
+                if (lane == 0) mbar_arrive(bar(C::BAR_PFULL + ti * 2 + sb));
             }
             // BAR_PVDONE cannot be used here: a parity wait cannot tell phase k from phase k-2, and
             // by now the barrier may be one or two phases ahead of what this thread last observed
-            if (ok) ok = mbar_wait_warp(bar(BAR_ALLDONE), 0, abort_flag);
+            if (ok) ok = mbar_wait_warp(bar(C::BAR_ALLDONE + ti), 0, abort_flag);
             if (ok) tc_fence_after();
             have_o = ok;
         }
@@ -408,34 +471,45 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             // ---------------------------------------------------------- partial rows to the workspace
             // straight from the registers of the TMEM read-out: element (chunk c, row r) of this
             // CTA's [32 chunks][128 rows] array of 16-byte chunks, so a warp stores 512 contiguous bytes
-            const long long cta_lin = ((long long)rt * gridDim.y + order) * S + rank;
+            const long long cta_lin = (((long long)blockIdx.z * NT + ti) * gridDim.y + order) * S + rank;
             float4 *my_o = reinterpret_cast<float4 *>(p.part_o + cta_lin * (MROWS * HD));
             float2 *my_ml = reinterpret_cast<float2 *>(p.part_ml + cta_lin * (MROWS * 2));
             if (have_o) {
-                // the whole row in one read-out (one wait instead of four), then 32 stores
-                uint32_t o[HD];
+                // the narrow shape reads the whole row out at once (one wait instead of four), the
+                // wide one, with fewer registers per thread, in two halves; 16-byte stores follow
+                constexpr int PIECE = NT == 1 ? HD : HD / 2;
+#pragma unroll 1
+                for (int c0 = 0; c0 < HD; c0 += PIECE) {
+                    uint32_t o[PIECE];
 #pragma unroll
-                for (int c4 = 0; c4 < HD / 32; ++c4) tmem_ld32(lane_base + TM_O + c4 * 32, o + c4 * 32);
-                tmem_ld_wait();
-                if (valid) {
+                    for (int c4 = 0; c4 < PIECE / 32; ++c4) tmem_ld32(lane_base + TM_O + c0 + c4 * 32, o + c4 * 32);
+                    tmem_ld_wait();
+                    if (valid) {
 #pragma unroll
-                    for (int c = 0; c < HD / 4; ++c)
-                        __stcg(my_o + c * MROWS + r,
-                               make_float4(__uint_as_float(o[c * 4]), __uint_as_float(o[c * 4 + 1]),
-                                           __uint_as_float(o[c * 4 + 2]), __uint_as_float(o[c * 4 + 3])));
+                        for (int c = 0; c < PIECE / 4; ++c)
+                            __stcg(my_o + (c0 / 4 + c) * MROWS + r,
+                                   make_float4(__uint_as_float(o[c * 4]), __uint_as_float(o[c * 4 + 1]),
+                                               __uint_as_float(o[c * 4 + 2]), __uint_as_float(o[c * 4 + 3])));
+                    }
                 }
             }
             // (a CTA without tiles has empty rows: sum 0, and its O rows are never read)
             if (valid) __stcg(my_ml + r, make_float2(have_o ? m_run : -INFINITY, have_o ? l_run : 0.f));
         }
         tc_fence_before();
-    } else if (warp == 4) {
+    } else if (warp == C::PRODUCER_WARP) {
         // ------------------------------------------------------------------ producer
         if (active && lane == 0) {
-            // the query rows of this tile: box = 64 columns x G heads x kb_rows positions
-            mbar_expect_tx(bar(BAR_QFULL), (uint32_t)(2 * 128 * p.G * kb_rows));
-            tma_load_4d(sbase + OFF_Q, &tm.q, 0, h * p.G, i0, b, bar(BAR_QFULL));
-            tma_load_4d(sbase + OFF_Q + QSUB_BYTES, &tm.q, 64, h * p.G, i0, b, bar(BAR_QFULL));
+            // the query rows of every tile: box = 64 columns x G heads x kb_rows positions
+            int n_q = 0;
+            for (int ti = 0; ti < NT; ++ti) n_q += tile_rows(ti) > 0;
+            mbar_expect_tx(bar(BAR_QFULL), (uint32_t)(n_q * 2 * 128 * p.G * kb_rows));
+            for (int ti = 0; ti < NT; ++ti)
+                if (tile_rows(ti) > 0) {
+                    const uint32_t q_dst = sbase + OFF_Q + ti * 2 * QSUB_BYTES;
+                    tma_load_4d(q_dst, &tm.q, 0, h * p.G, tile_i0(ti), b, bar(BAR_QFULL));
+                    tma_load_4d(q_dst + QSUB_BYTES, &tm.q, 64, h * p.G, tile_i0(ti), b, bar(BAR_QFULL));
+                }
             bool ok = true;
             const int n_items = 2 * n_tiles;
             while (produced < n_items && ok) {
@@ -453,11 +527,12 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                 mbar_wait(bar(BAR_QFULL), 0, &dummy);
             }
         }
-    } else if (active) {
-        // ------------------------------------------------------------------ MMA issue
-        const uint32_t q_addr = sbase + OFF_Q;
+    } else if (active && tile_rows(warp - C::MMA_WARP) > 0) {
+        // ------------------------------------------------------------------ MMA issue, query tile ti
+        const int ti = warp - C::MMA_WARP;
         constexpr uint32_t IDESC_QK = make_idesc(TN, 0);      // A = Q, B = K tile, both K-major
         constexpr uint32_t IDESC_PV = make_idesc(HD, 1);      // A = P (TMEM), B = V tile (MN-major)
+        const uint32_t q_addr = sbase + OFF_Q + ti * 2 * QSUB_BYTES;
         auto issue_qk = [&](int t) -> bool {
             const int j = item_of_k(t), slot = j % NSLOT;
             if (!mbar_wait_warp(bar(BAR_FULL + slot), (j / NSLOT) & 1, abort_flag)) return false;
@@ -466,13 +541,13 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                 const uint32_t k_addr = sbase + OFF_RING + slot * SLOT_BYTES;
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {        // 16 head-dim columns per MMA
-                    umma_ss(tmem + TM_S + (t & 1) * TN,
+                    umma_ss(tmem + C::tm_s(ti, t & 1),
                             make_desc(q_addr + (kk >> 2) * QSUB_BYTES + (kk & 3) * 32, 16, 1024),
                             make_desc(k_addr + (kk >> 2) * SUB_BYTES + (kk & 3) * 32, 16, 1024),
                             IDESC_QK, kk > 0);
                 }
                 umma_commit(bar(BAR_EMPTY + slot));
-                umma_commit(bar(BAR_SFULL + (t & 1)));
+                umma_commit(bar(C::BAR_SFULL + ti * 2 + (t & 1)));
             }
             __syncwarp();
             return true;
@@ -481,7 +556,8 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             const int j = item_of_v(t), slot = j % NSLOT;
             if (!mbar_wait_warp(bar(BAR_FULL + slot), (j / NSLOT) & 1, abort_flag)) return false;
             // a ragged prefix tile: V rows past the prefix may hold anything, and 0 * NaN would
-            // poison the product, so they are cleared before the MMA reads them
+            // poison the product, so they are cleared before the MMA reads them (by every MMA
+            // warp: the same zeros, and no warp has to wait for another)
             const int nv = t < n_mine ? min(TN, P - ((int)t0 + t) * TN) : (p.blk_in_cache ? p.K : TN);
             if (nv < TN) {
                 unsigned char *vt = smem + OFF_RING + slot * SLOT_BYTES;
@@ -492,18 +568,18 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                 fence_proxy_async();
                 __syncwarp();
             }
-            if (!mbar_wait_warp(bar(BAR_PFULL + (t & 1)), (t >> 1) & 1, abort_flag)) return false;
+            if (!mbar_wait_warp(bar(C::BAR_PFULL + ti * 2 + (t & 1)), (t >> 1) & 1, abort_flag)) return false;
             tc_fence_after();
             if (lane == 0) {
                 const uint32_t v_addr = sbase + OFF_RING + slot * SLOT_BYTES;
 #pragma unroll
                 for (int kk = 0; kk < TN / 16; ++kk) {        // 16 key positions per MMA
-                    umma_ts(tmem + TM_O, tmem + TM_S + (t & 1) * TN + kk * 8,
+                    umma_ts(tmem + C::tm_o(ti), tmem + C::tm_s(ti, t & 1) + kk * 8,
                             make_desc(v_addr + kk * 2048, SUB_BYTES, 1024), IDESC_PV, (t > 0) || (kk > 0));
                 }
                 umma_commit(bar(BAR_EMPTY + slot));
-                umma_commit(bar(BAR_PVDONE));
-                if (t == n_tiles - 1) umma_commit(bar(BAR_ALLDONE));
+                umma_commit(bar(C::BAR_PVDONE + ti));
+                if (t == n_tiles - 1) umma_commit(bar(C::BAR_ALLDONE + ti));
             }
             __syncwarp();
             return true;
@@ -514,42 +590,31 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             if (t + 1 < n_tiles) ok = issue_qk(t + 1);
             if (ok) ok = issue_pv(t);
         }
-        // every MMA must have retired before TMEM is freed
-        if (ok) mbar_wait_warp(bar(BAR_ALLDONE), 0, abort_flag);
+        // every MMA of this warp must have retired before TMEM is freed
+        if (ok) mbar_wait_warp(bar(C::BAR_ALLDONE + ti), 0, abort_flag);
         tc_fence_before();
     }
 
     // ---------------------------------------------------------------------- merge
     __syncthreads();
     tc_fence_after();
-    if (warp == 5)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TM_COLS) : "memory");
+    if (warp == C::MMA_WARP)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::TM_COLS) : "memory");
     if (tid == 0 && *abort_flag && p.status) atomicOr(p.status, ORTHRUS_DEV_WAIT_TIMEOUT);
     if (S == 1) return;
     constexpr int NWARPS = NTHREADS / 32;
-    auto out_row = [&](int R) {
-        const int i = i0 + R / p.G, g = R % p.G;
-        return static_cast<__nv_bfloat16 *>(p.out) + (((long long)b * p.K + i) * p.Hq + h * p.G + g) * HD;
-    };
-    {
-        // The cluster is what guarantees that the CTAs waiting for one another are resident
-        // together.  Release / acquire at cluster scope: every CTA's partial rows are in place.
-        cluster_sync_all();
-        const long long grp_lin = ((long long)rt * gridDim.y + order) * S;
-        const float4 *grp_o = reinterpret_cast<const float4 *>(p.part_o + grp_lin * (MROWS * HD));
-        const float2 *grp_ml = reinterpret_cast<const float2 *>(p.part_ml + grp_lin * (MROWS * 2));
-        const int n_tasks = ((rows_here + 31) >> 5) * (HD / 4);
-        auto run = [&](auto sp) {
-            l2_merge_tasks<decltype(sp)::value>(S, rank, warp, lane, NWARPS, n_tasks, rows_here, grp_o, grp_ml,
-                                                [&](int R, int c, const float4 &acc, float inv) {
-                reinterpret_cast<uint2 *>(out_row(R))[c] =
-                    make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
-            });
-        };
-        if (S <= 2) run(std::integral_constant<int, 2>());
-        else if (S <= 4) run(std::integral_constant<int, 4>());
-        else if (S <= 8) run(std::integral_constant<int, 8>());
-        else run(std::integral_constant<int, 16>());
+    // The cluster is what guarantees that the CTAs waiting for one another are resident
+    // together.  Release / acquire at cluster scope: every CTA's partial rows are in place.
+    cluster_sync_all();
+    for (int ti = 0; ti < NT; ++ti) {
+        const int rows_here = tile_rows(ti);
+        if (rows_here == 0) break;
+        __nv_bfloat16 *out_tile = static_cast<__nv_bfloat16 *>(p.out) +
+                                  (((long long)b * p.K + tile_i0(ti)) * p.Hq + h * p.G) * HD;
+        const long long grp_lin = (((long long)blockIdx.z * NT + ti) * gridDim.y + order) * S;
+        merge_tile<NT == 1 ? 16 : 8>(S, rank, warp, lane, NWARPS, rows_here,
+                   reinterpret_cast<const float4 *>(p.part_o + grp_lin * (MROWS * HD)),
+                   reinterpret_cast<const float2 *>(p.part_ml + grp_lin * (MROWS * 2)), out_tile, p.G, p.Hq);
     }
 }
 
@@ -632,35 +697,76 @@ int tc_row_tiles(int G, int K)
     return (K + kb - 1) / kb;
 }
 
+// Query tiles per CTA: units wider than one 128-row tile take the shape whose two query tiles share
+// one K/V ring (the cache is then streamed once per pair of tiles instead of once per tile).
+// ORTHRUS_TC_ROW_TILES_PER_CTA=1 keeps the narrow shape, for measurements.
+int tc_tiles_per_cta(int G, int K)
+{
+    static const int forced = [] { const char *e = getenv("ORTHRUS_TC_ROW_TILES_PER_CTA"); return e ? atoi(e) : 0; }();
+    if (forced == 1 || forced == 2) return tc_row_tiles(G, K) >= 2 ? forced : 1;
+    return tc_row_tiles(G, K) >= 2 ? 2 : 1;
+}
+
+// CTAs along the query-tile axis of the grid
+int tc_cta_groups(int G, int K)
+{
+    const int nt = tc_tiles_per_cta(G, K);
+    return (tc_row_tiles(G, K) + nt - 1) / nt;
+}
+
 bool tc_driver_ok() { return encode_fn() != nullptr; }
 
-// CTAs of this kernel one SM of the current device keeps resident: what its shared memory holds
-// (each CTA also costs the 1 KB the system reserves per block), at most the two that share
-// the 512 TMEM columns.  2 on a B200.  Asked once per device; 2 assumed where there is none.
-int tc_ctas_per_sm()
+// CTAs of the shape with nt query tiles one SM of the current device keeps resident: what its
+// shared memory holds (each CTA also costs the 1 KB the system reserves per block), at most what
+// the 512 TMEM columns allow.  2 and 1 on a B200.  Asked once per device; those values are assumed
+// where there is no device.
+int tc_ctas_per_sm(int nt)
 {
     constexpr int kMaxDevices = 64;
     static std::mutex mu;
-    static int cached[kMaxDevices] = {};
+    static int smem_cached[kMaxDevices] = {};
+    const int smem_bytes = nt == 2 ? Shape<2>::SMEM_BYTES : Shape<1>::SMEM_BYTES;
+    const int by_tmem = nt == 2 ? 1 : 2;
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { (void)cudaGetLastError(); return 2; }
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { (void)cudaGetLastError(); return by_tmem; }
     std::lock_guard<std::mutex> lock(mu);
-    if (cached[dev]) return cached[dev];
-    int smem_per_sm = 0;
-    if (cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return 2;
+    if (!smem_cached[dev]) {
+        int smem_per_sm = 0;
+        if (cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return by_tmem;
+        }
+        smem_cached[dev] = smem_per_sm;
     }
-    int n = smem_per_sm / (SMEM_BYTES + 1024);
-    n = n < 1 ? 1 : (n > 512 / (int)TM_COLS ? 512 / (int)TM_COLS : n);
-    cached[dev] = n;
-    return n;
+    const int n = smem_cached[dev] / (smem_bytes + 1024);
+    return n < 1 ? 1 : (n > by_tmem ? by_tmem : n);
 }
 
-// Largest cluster size (a power of two up to 16) the current device can co-schedule for this
-// kernel; 16 on a full B200.  Without a device (or if the query fails) 16 is assumed and a
-// launch that cannot be scheduled reports its error.
-int tc_max_cluster()
+namespace {
+
+template <int NT>
+cudaError_t configure_kernel()
+{   // function attributes belong to a device: set them once on each device that launches
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static bool configured[kMaxDevices] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!configured[dev]) {
+        e = cudaFuncSetAttribute(attend_tc_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, Shape<NT>::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attend_tc_kernel<NT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    return cudaSuccess;
+}
+
+template <int NT>
+int max_cluster_of_shape()
 {
     constexpr int kMaxDevices = 64;
     static std::mutex mu;
@@ -670,19 +776,18 @@ int tc_max_cluster()
     std::lock_guard<std::mutex> lock(mu);
     if (cached[dev]) return cached[dev];
     int best = 16;
-    if (cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) == cudaSuccess &&
-        cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+    if (configure_kernel<NT>() == cudaSuccess) {
         for (int s = 16; s >= 2; s >>= 1) {
             cudaLaunchConfig_t cfg = {};
             cfg.gridDim = dim3(s, 1, 1);
-            cfg.blockDim = dim3(NTHREADS);
-            cfg.dynamicSmemBytes = SMEM_BYTES;
+            cfg.blockDim = dim3(Shape<NT>::NTHREADS);
+            cfg.dynamicSmemBytes = Shape<NT>::SMEM_BYTES;
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeClusterDimension;
             attr[0].val.clusterDim.x = s; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
             cfg.attrs = attr; cfg.numAttrs = 1;
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, attend_tc_kernel, &cfg) == cudaSuccess && n > 0) { best = s; break; }
+            if (cudaOccupancyMaxActiveClusters(&n, attend_tc_kernel<NT>, &cfg) == cudaSuccess && n > 0) { best = s; break; }
             best = s >> 1;
         }
         if (best < 1) best = 1;
@@ -692,31 +797,26 @@ int tc_max_cluster()
     cached[dev] = best;
     return best;
 }
+
+}  // namespace
+
+// Largest cluster size (a power of two up to 16) the current device can co-schedule for the shape
+// with nt query tiles; 16 on a full B200.  Without a device (or if the query fails) 16 is assumed
+// and a launch that cannot be scheduled reports its error.
+int tc_max_cluster(int nt) { return nt == 2 ? max_cluster_of_shape<2>() : max_cluster_of_shape<1>(); }
 int tc_tile_positions() { return TN; }
+
+template <int NT>
 static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int flags, cudaStream_t st)
 {
     const int S = p.n_splits;
-    {   // function attributes belong to a device: set them once on each device that launches
-        constexpr int kMaxDevices = 64;
-        static std::mutex mu;
-        static bool configured[kMaxDevices] = {};
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-        std::lock_guard<std::mutex> lock(mu);
-        if (!configured[dev]) {
-            e = cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-            if (e == cudaSuccess)
-                e = cudaFuncSetAttribute(attend_tc_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-            if (e != cudaSuccess) return e;
-            configured[dev] = true;
-        }
-    }
+    cudaError_t e = configure_kernel<NT>();
+    if (e != cudaSuccess) return e;
+    const int row_tiles = (p.K + kb - 1) / kb;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(S, p.B * p.Hkv, (p.K + kb - 1) / kb);
-    cfg.blockDim = dim3(NTHREADS);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.gridDim = dim3(S, p.B * p.Hkv, (row_tiles + NT - 1) / NT);
+    cfg.blockDim = dim3(Shape<NT>::NTHREADS);
+    cfg.dynamicSmemBytes = Shape<NT>::SMEM_BYTES;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     int n_attr = 0;
@@ -734,8 +834,7 @@ static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int 
     }
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, attend_tc_kernel, p, tm, S, kb,
-                                       (flags & ORTHRUS_LAYER_CACHE_QUIESCENT) ? 1 : 0);
+    e = cudaLaunchKernelEx(&cfg, attend_tc_kernel<NT>, p, tm, S, kb, (flags & ORTHRUS_LAYER_CACHE_QUIESCENT) ? 1 : 0);
     count_launch();
     return e;
 }
@@ -753,7 +852,7 @@ cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st)
     } else if (!get_map(p.k_blk, p.Hkv, p.K, p.B, 1, TN, &tm.kb) || !get_map(p.v_blk, p.Hkv, p.K, p.B, 1, TN, &tm.vb)) {
         return cudaErrorInvalidValue;
     }
-    return launch_tc(p, tm, kb, flags, st);
+    return tc_tiles_per_cta(p.G, p.K) == 2 ? launch_tc<2>(p, tm, kb, flags, st) : launch_tc<1>(p, tm, kb, flags, st);
 }
 
 }  // namespace orthrus

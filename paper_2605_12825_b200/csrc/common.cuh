@@ -73,8 +73,10 @@ int mma_tile_positions();
 bool tc_driver_ok();                    // the driver offers cuTensorMapEncodeTiled
 cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st);   // n_splits = cluster size
 int tc_row_tiles(int G, int K);          // 128-row query tiles per unit (0: group too wide)
-int tc_ctas_per_sm();
-int tc_max_cluster();                   // largest cluster the device can co-schedule (<= 16)
+int tc_tiles_per_cta(int G, int K);      // query tiles that share one K/V ring in a CTA (1 or 2)
+int tc_cta_groups(int G, int K);         // CTAs along the query-tile axis: ceil(row tiles / tiles per CTA)
+int tc_ctas_per_sm(int nt);              // resident CTAs per SM of the shape with nt query tiles
+int tc_max_cluster(int nt);              // largest cluster the device can co-schedule (<= 16)
 int tc_tile_positions();
 cudaError_t launch_combine(const AttnParams &p, int dtype, cudaStream_t st);
 
