@@ -127,8 +127,10 @@ enum {
 size_t orthrus_attend_workspace_bytes(const orthrus_layer_t *layer);
 
 /*
- * Zeroes the workspace header (status word).  Call once after allocating a
- * workspace and whenever the status word should be cleared.
+ * Zeroes the workspace: the status word in its header, and the arrival counters the
+ * attention kernels keep in it (they return to zero at the end of every call that
+ * completes).  Call once after allocating a workspace, whenever the status word should
+ * be cleared, and after a call that reported ORTHRUS_DEV_WAIT_TIMEOUT.
  */
 orthrus_status_t orthrus_workspace_init(void *workspace, size_t workspace_bytes, void *stream);
 

@@ -112,6 +112,19 @@ static bool tc_usable(const orthrus_layer_t *L)
     return rows < 0x7fffffffull && tc_driver_ok();
 }
 
+// ORTHRUS_TC_SCHEDULE=stream (read at every call) selects the persistent kernel, which cuts the
+// work by tiles instead of by units, for the shapes it serves; it was measured slower than the
+// cluster kernel and is a measurement knob.  A forced split count keeps the cluster kernel.
+static bool tc_use_stream(const orthrus_layer_t *L)
+{
+    if (!tc_usable(L)) return false;
+    const int G = L->n_q_heads / L->n_kv_heads;
+    if (!tc_stream_shape(L->batch, G, L->block) || env_int("ORTHRUS_SPLITS", 0) > 0) return false;
+    const char *e = getenv("ORTHRUS_TC_SCHEDULE");
+    return e && !strcmp(e, "stream");
+}
+static int tc_stream_ctas() { return tc_ctas_per_sm(1) * num_sms(); }
+
 static Plan make_plan(const orthrus_layer_t *L, bool tc)
 {
     const int max_len = max_len_of(L);
@@ -197,9 +210,12 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
         return ORTHRUS_ERR_INVALID_ARG;
     const int want = current_path();
     const bool tc = (want == PATH_AUTO || want == PATH_TCGEN05) && tc_usable(L);
-    const Plan pl = make_plan(L, tc);
+    const bool stream_k = tc && tc_use_stream(L);
+    Plan pl = make_plan(L, tc);
+    if (stream_k) pl.n_splits = 1;
     size_t ml_off = 0;
-    const size_t need = kHeaderBytes + partial_bytes(L, pl, &ml_off, tc);
+    const size_t need = kHeaderBytes + (stream_k ? tc_stream_workspace_bytes(L->batch, L->n_kv_heads, tc_stream_ctas())
+                                                 : partial_bytes(L, pl, &ml_off, tc));
     if (ws_bytes < need) return ORTHRUS_ERR_WORKSPACE;
 
     AttnParams p;
@@ -224,7 +240,8 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
         t_last_path = "tcgen05";
         int flags = (int)(L->flags & (ORTHRUS_LAYER_CACHE_QUIESCENT | ORTHRUS_LAYER_NO_EARLY_LAUNCH));
         if (env_int("ORTHRUS_NO_EARLY_LAUNCH", 0)) flags |= ORTHRUS_LAYER_NO_EARLY_LAUNCH;
-        e = launch_attend_tc(p, flags, cs);
+        if (stream_k) e = launch_attend_tc_stream(p, tc_stream_ctas(), base + kHeaderBytes, flags, cs);
+        else e = launch_attend_tc(p, flags, cs);
         merge_kernel = false;
     } else if (want != PATH_SIMT && mma_path_supports(p, L->dtype)) {
         t_last_path = "mma";
@@ -255,6 +272,10 @@ size_t orthrus_attend_workspace_bytes(const orthrus_layer_t *layer)
     if (tc_usable(layer)) {
         const size_t n2 = partial_bytes(layer, make_plan(layer, true), nullptr, true);
         if (n2 > need) need = n2;
+        if (tc_use_stream(layer)) {
+            const size_t n3 = tc_stream_workspace_bytes(layer->batch, layer->n_kv_heads, tc_stream_ctas());
+            if (n3 > need) need = n3;
+        }
     }
     return kHeaderBytes + need;
 }
@@ -262,7 +283,8 @@ size_t orthrus_attend_workspace_bytes(const orthrus_layer_t *layer)
 orthrus_status_t orthrus_workspace_init(void *workspace, size_t workspace_bytes, void *stream)
 {
     if (!workspace || workspace_bytes < (size_t)kHeaderBytes) return ORTHRUS_ERR_INVALID_ARG;
-    return cudaMemsetAsync(workspace, 0, kHeaderBytes, static_cast<cudaStream_t>(stream)) == cudaSuccess
+    // all of it: besides the status word, the arrival counters some kernels keep there must start at zero
+    return cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
 }
 

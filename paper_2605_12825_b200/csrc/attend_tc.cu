@@ -618,6 +618,8 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     }
 }
 
+#include "attend_tc_stream.cuh"
+
 // ---------------------------------------------------------------------------- host side
 
 }  // namespace
@@ -836,6 +838,68 @@ static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int 
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
     e = cudaLaunchKernelEx(&cfg, attend_tc_kernel<NT>, p, tm, S, kb, (flags & ORTHRUS_LAYER_CACHE_QUIESCENT) ? 1 : 0);
+    count_launch();
+    return e;
+}
+
+// The persistent kernel serves one query tile per unit and ranks at most 128 batch entries.
+bool tc_stream_shape(int B, int G, int K) { return B <= STREAM_MAX_B && G >= 1 && G * K <= MROWS && K <= TN; }
+
+// Workspace of the persistent kernel behind the header: two partial tiles and their (max, sum)
+// rows per CTA, then one arrival counter per unit (zero between calls).
+size_t tc_stream_workspace_bytes(int B, int Hkv, int n_ctas)
+{
+    return (size_t)n_ctas * 2 * (MROWS * HD * sizeof(float) + MROWS * 2 * sizeof(float)) +
+           (((size_t)B * Hkv * sizeof(int32_t) + 255) / 256) * 256;
+}
+
+cudaError_t launch_attend_tc_stream(const AttnParams &p, int n_ctas, void *ws_body, int flags, cudaStream_t st)
+{
+    TcMaps tm;
+    const unsigned long long rows = (unsigned long long)(p.B / p.nb) * p.Hkv * p.capacity;
+    if (!get_map(p.k_cache, rows, 0, 0, TN, 0, &tm.k) || !get_map(p.v_cache, rows, 0, 0, TN, 0, &tm.v) ||
+        !get_map(p.q, p.Hq, p.K, p.B, p.G, p.K, &tm.q))
+        return cudaErrorInvalidValue;
+    if (p.blk_in_cache) {
+        tm.kb = tm.k; tm.vb = tm.v;
+    } else if (!get_map(p.k_blk, p.Hkv, p.K, p.B, 1, TN, &tm.kb) || !get_map(p.v_blk, p.Hkv, p.K, p.B, 1, TN, &tm.vb)) {
+        return cudaErrorInvalidValue;
+    }
+    {   // function attributes belong to a device: set them once on each device that launches
+        constexpr int kMaxDevices = 64;
+        static std::mutex mu;
+        static bool configured[kMaxDevices] = {};
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> lock(mu);
+        if (!configured[dev]) {
+            e = cudaFuncSetAttribute(attend_tc_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, STREAM_SMEM_BYTES);
+            if (e != cudaSuccess) return e;
+            configured[dev] = true;
+        }
+    }
+    StreamArgs sa;
+    unsigned char *base = static_cast<unsigned char *>(ws_body);
+    sa.part_o = reinterpret_cast<float4 *>(base);
+    sa.part_ml = reinterpret_cast<float2 *>(base + (size_t)n_ctas * 2 * MROWS * HD * sizeof(float));
+    sa.counters = reinterpret_cast<int32_t *>(base + (size_t)n_ctas * 2 * (MROWS * HD + MROWS * 2) * sizeof(float));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_ctas, 1, 1);
+    cfg.blockDim = dim3(Shape<1>::NTHREADS);
+    cfg.dynamicSmemBytes = STREAM_SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    int n_attr = 0;
+    if (!(flags & ORTHRUS_LAYER_NO_EARLY_LAUNCH)) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n_attr;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, attend_tc_stream_kernel, p, tm, sa);
     count_launch();
     return e;
 }

@@ -78,6 +78,9 @@ int tc_cta_groups(int G, int K);         // CTAs along the query-tile axis: ceil
 int tc_ctas_per_sm(int nt);              // resident CTAs per SM of the shape with nt query tiles
 int tc_max_cluster(int nt);              // largest cluster the device can co-schedule (<= 16)
 int tc_tile_positions();
+bool tc_stream_shape(int B, int G, int K);                  // the persistent kernel serves this shape
+size_t tc_stream_workspace_bytes(int B, int Hkv, int n_ctas);
+cudaError_t launch_attend_tc_stream(const AttnParams &p, int n_ctas, void *ws_body, int flags, cudaStream_t st);
 cudaError_t launch_combine(const AttnParams &p, int dtype, cudaStream_t st);
 
 cudaError_t launch_consensus(const void *logits, int dtype, const int32_t *draft, int B, int K,
