@@ -365,6 +365,39 @@ def read_bandwidth_probe(dev, stream) -> float:
     return best
 
 
+def sustained_probes(dev, stream, gpu_index, seconds=0.5):
+    """The same two library kernels the burst denominators come from (a copy, a reduction), run back
+    to back for `seconds` with the clocks sampled: what plain streaming sustains on this GPU, as
+    context for the long timed regions of the long-prefix workloads (which reach the power limit)."""
+    n = 1 << 29
+    a = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    b = torch.empty_like(a)
+    a.fill_(1.0)
+    out = {}
+    for name, fn, nbytes in (("copy", lambda: b.copy_(a), 4.0 * n), ("read", lambda: a.sum(dtype=torch.float32), 2.0 * n)):
+        for _ in range(3):
+            fn()
+        stream.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fn()
+        e1.record(stream)
+        stream.synchronize()
+        reps = max(10, int(seconds * 1e3 / max(e0.elapsed_time(e1), 1e-3)))
+        sampler = ClockSampler(gpu_index)
+        sampler.start()
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        stream.synchronize()
+        clocks = sampler.stop()
+        out[name] = {"gbs": round(nbytes * reps / (e0.elapsed_time(e1) * 1e-3) / 1e9, 1), "repetitions": reps,
+                     "clocks": {k: clocks.get(k) for k in ("sm_mhz", "samples", "reasons")}}
+    del a, b
+    return out
+
+
 def capture(fn, stream):
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g, stream=stream):
@@ -744,6 +777,8 @@ def run_gpu(args):
     if world == 1 and not args.no_extra_workloads and args.workload == DEFAULT_WORKLOAD and not args.block:
         # the long-prefix and loop-shaped workloads on the same line: the bandwidth target is
         # stated on these, the headline value stays the one above
+        with torch.cuda.stream(stream):
+            out["sustained_probes"] = sustained_probes(dev, stream, local)
         out["workloads"] = {}
         for name in ("cfg3_ragged", "cfg4_long", "cfg5_loop"):
             out["workloads"][name] = workload_entry(B, name, dev, stream, flags, max(3, min(args.steps, 30)),
