@@ -634,6 +634,65 @@ def workload_entry(B, name, dev, stream, flags, steps, gpu_index, peak, min_regi
     return out
 
 
+def multi_block_entry(B, dev, stream, reps=20):
+    """The multi-block mask of Eq. 6 on a training-shaped call (8B head layout, 4 sequences of 4096
+    clean positions, 32 anchored blocks of 8 each, anchors increasing along a sequence): the form
+    whose blocks share 128-row query tiles against one unit per block, L2 flushed before each call;
+    four blocks of sequence 0 against the oracle."""
+    import oracle
+    oracle.build()
+    S, NB, K, Hq, Hkv, d, L = 4, 32, 8, 32, 8, 128, 4096
+    g = torch.Generator().manual_seed(11)
+    cap = L + 64
+    mk = lambda *sh: (torch.randn(*sh, generator=g) * 0.7).to(torch.bfloat16)
+    host = dict(q=mk(S, NB, K, Hq, d), k_blk=mk(S, NB, K, Hkv, d), v_blk=mk(S, NB, K, Hkv, d),
+                k_cache=mk(S, Hkv, cap, d), v_cache=mk(S, Hkv, cap, d),
+                cache_len=torch.full((S,), L, dtype=torch.int32),
+                anchors=torch.randint(0, L + 1, (S, NB), generator=g).sort(dim=1).values.to(torch.int32).contiguous())
+    t = {k: v.to(dev) for k, v in host.items()}
+    layer = B.make_layer(t["k_cache"], t["v_cache"], t["cache_len"], Hq, K, L)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    res = {"shape": {"sequences": S, "blocks": NB, "block": K, "n_q_heads": Hq, "n_kv_heads": Hkv, "head_dim": d,
+                     "clean_len": L},
+           "requested_bytes": int(host["anchors"].sum()) * Hkv * d * 2 * 2 + 4 * S * NB * K * (Hq + Hkv) * d,
+           "distinct_bytes": int(host["anchors"].max(dim=1).values.sum()) * Hkv * d * 2 * 2 + 4 * S * NB * K * (Hq + Hkv) * d}
+    saved = os.environ.pop("ORTHRUS_MULTI_BLOCK_PACK", None)
+    try:
+        for key, pack in (("shared_tiles_us", "1"), ("unit_per_block_us", "0")):
+            os.environ["ORTHRUS_MULTI_BLOCK_PACK"] = pack
+            ws = B.new_workspace(B.orthrus_multi_block_workspace_bytes(layer, NB), device=dev)
+            out = torch.empty_like(t["q"])
+            ts = []
+            for it in range(reps + 3):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                B.orthrus_multi_block_attend(layer, t["anchors"], t["q"], t["k_blk"], t["v_blk"], out, ws, stream)
+                e1.record(stream)
+                stream.synchronize()
+                if it >= 3:
+                    ts.append(e0.elapsed_time(e1) * 1e3)
+            if B.orthrus_read_status(ws, stream) != 0:
+                raise SystemExit("bench.py: multi-block call left a device status")
+            res[key] = round(statistics.median(ts), 2)
+            pick = torch.tensor([0, 10, 21, 31])
+            ref = oracle.multi_block_attend(host["q"][:1, pick].contiguous(), host["k_blk"][:1, pick].contiguous(),
+                                            host["v_blk"][:1, pick].contiguous(), host["k_cache"][:1].contiguous(),
+                                            host["v_cache"][:1].contiguous(), host["cache_len"][:1].contiguous(),
+                                            host["anchors"][:1, pick].contiguous())
+            err = float((out[:1].cpu()[:, pick].double() - ref).abs().max())
+            scale = float(ref.abs().max())
+            if not (err <= 2e-2 and err <= 1e-2 * scale):
+                raise SystemExit(f"bench.py: multi-block output is off the oracle (max-abs {err:.3e}, max|ref| {scale:.3e})")
+            res[key.replace("_us", "_max_err_over_max_ref")] = round(err / scale, 5)
+    finally:
+        os.environ.pop("ORTHRUS_MULTI_BLOCK_PACK", None)
+        if saved is not None:
+            os.environ["ORTHRUS_MULTI_BLOCK_PACK"] = saved
+    res["launches"] = 2 * (reps + 3)
+    return res
+
+
 def run_gpu(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -783,6 +842,9 @@ def run_gpu(args):
         for name in ("cfg3_ragged", "cfg4_long", "cfg5_loop"):
             out["workloads"][name] = workload_entry(B, name, dev, stream, flags, max(3, min(args.steps, 30)),
                                                     local, peak)
+        with torch.cuda.stream(stream):
+            out["multi_block_eq6"] = multi_block_entry(B, dev, stream)
+        torch.cuda.empty_cache()
     cycles = args.decoder_cycles
     if world == 1 and (cycles > 0 or (cycles == 0 and not args.no_extra_workloads and
                                       args.workload == DEFAULT_WORKLOAD and not args.block)):

@@ -171,7 +171,11 @@ orthrus_status_t orthrus_ar_verify_attend(const orthrus_layer_t *layer,
  *                          outside are clamped and flagged like a bad cache_len); the caller
  *                          keeps them at or below the sequence's clean length
  * layer describes the S sequences (batch = S; cache_len is not read; max_len_hint bounds
- * the anchors).  Blocks are independent units of work, scheduled longest prefix first.
+ * the anchors).  On the tcgen05 path, when at least two blocks fit the 128 rows of a query
+ * tile (2 * K * Hq/Hkv <= 128), consecutive blocks of a sequence share query tiles: the
+ * prefix is streamed once per tile, up to the largest anchor among its blocks, each row
+ * masked at its own anchor and to its own block's keys.  Otherwise every block is a unit
+ * of work of its own, scheduled longest prefix first.
  * Workspace: orthrus_multi_block_workspace_bytes(layer, n_blocks).
  */
 size_t orthrus_multi_block_workspace_bytes(const orthrus_layer_t *layer, int32_t n_blocks);

@@ -229,7 +229,7 @@ static orthrus_status_t attend(const orthrus_layer_t *L, int causal, const void 
     p.G = p.Hq / p.Hkv; p.M = p.G * p.K; p.d = L->head_dim; p.capacity = L->capacity;
     p.chunk = pl.chunk; p.n_splits = pl.n_splits; p.causal = causal;
     p.blk_in_cache = in_cache ? 1 : 0;
-    p.nb = nb; p.len_cap = L->capacity - L->block;
+    p.nb = nb; p.kb_width = 0; p.len_cap = L->capacity - L->block;
     const float scale = L->softmax_scale > 0.f ? L->softmax_scale : 1.f / sqrtf((float)p.d);
     p.scale_log2 = scale * 1.4426950408889634f;
 
@@ -315,11 +315,76 @@ static bool multi_block_layer(const orthrus_layer_t *layer, int32_t n_blocks, co
     return true;
 }
 
+// The packed form of Eq. 6 (tcgen05 path): the blocks of a sequence share 128-row query tiles, so
+// the prefix is streamed once per tile instead of once per block.  Taken when at least two blocks
+// fit one tile; ORTHRUS_MULTI_BLOCK_PACK=0 keeps the one-unit-per-block form (a measurement knob).
+static bool multi_block_packed(const orthrus_layer_t *layer, int32_t n_blocks)
+{
+    if (n_blocks < 2 || check_layer(layer) != ORTHRUS_OK || !tc_usable(layer)) return false;
+    const int want = current_path();
+    if (want != PATH_AUTO && want != PATH_TCGEN05) return false;
+    if (2 * (layer->n_q_heads / layer->n_kv_heads) * layer->block > 128) return false;
+    if ((long long)n_blocks * layer->block > (1 << 20)) return false;
+    const char *e = getenv("ORTHRUS_MULTI_BLOCK_PACK");
+    return !(e && e[0] == '0');
+}
+
+// the descriptor the packed form plans with: one "block" of n_blocks * K positions per sequence
+static orthrus_layer_t packed_layer(const orthrus_layer_t *layer, int32_t n_blocks)
+{
+    orthrus_layer_t L = *layer;
+    L.max_len_hint = max_len_of(layer);
+    L.block = n_blocks * layer->block;
+    L.flags = layer->flags & ~(uint32_t)ORTHRUS_LAYER_BLOCK_IN_CACHE;
+    return L;
+}
+
+static orthrus_status_t attend_packed(const orthrus_layer_t *layer, int32_t n_blocks, const int32_t *anchors,
+                                      const void *q, const void *k_blk, const void *v_blk, void *out,
+                                      void *ws, size_t ws_bytes, void *stream)
+{
+    if (!q || !k_blk || !v_blk || !out || !ws || !layer->k_cache || !layer->v_cache) return ORTHRUS_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out) || !aligned16(ws) ||
+        !aligned16(layer->k_cache) || !aligned16(layer->v_cache) || (reinterpret_cast<uintptr_t>(anchors) & 3))
+        return ORTHRUS_ERR_INVALID_ARG;
+    const orthrus_layer_t L = packed_layer(layer, n_blocks);
+    const Plan pl = make_plan(&L, true);
+    size_t ml_off = 0;
+    if (ws_bytes < kHeaderBytes + partial_bytes(&L, pl, &ml_off, true)) return ORTHRUS_ERR_WORKSPACE;
+
+    AttnParams p;
+    p.q = q; p.k_blk = k_blk; p.v_blk = v_blk; p.k_cache = layer->k_cache; p.v_cache = layer->v_cache;
+    p.cache_len = anchors; p.out = out;
+    unsigned char *base = static_cast<unsigned char *>(ws);
+    p.status = reinterpret_cast<int32_t *>(base);
+    p.part_o = reinterpret_cast<float *>(base + kHeaderBytes);
+    p.part_ml = reinterpret_cast<float *>(base + kHeaderBytes + ml_off);
+    p.B = layer->batch; p.K = L.block; p.Hq = layer->n_q_heads; p.Hkv = layer->n_kv_heads;
+    p.G = p.Hq / p.Hkv; p.M = p.G * p.K; p.d = layer->head_dim; p.capacity = layer->capacity;
+    p.chunk = pl.chunk; p.n_splits = pl.n_splits; p.causal = 0; p.blk_in_cache = 0;
+    p.nb = n_blocks; p.kb_width = layer->block; p.len_cap = layer->capacity - layer->block;
+    const float scale = layer->softmax_scale > 0.f ? layer->softmax_scale : 1.f / sqrtf((float)p.d);
+    p.scale_log2 = scale * 1.4426950408889634f;
+    t_last_path = "tcgen05";
+    int flags = (int)(layer->flags & (ORTHRUS_LAYER_CACHE_QUIESCENT | ORTHRUS_LAYER_NO_EARLY_LAUNCH));
+    if (env_int("ORTHRUS_NO_EARLY_LAUNCH", 0)) flags |= ORTHRUS_LAYER_NO_EARLY_LAUNCH;
+    return launch_attend_tc_packed(p, flags, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? ORTHRUS_OK : ORTHRUS_ERR_CUDA;
+}
+
 size_t orthrus_multi_block_workspace_bytes(const orthrus_layer_t *layer, int32_t n_blocks)
 {
     orthrus_layer_t L;
     if (!multi_block_layer(layer, n_blocks, nullptr, &L)) return 0;
-    return orthrus_attend_workspace_bytes(&L);
+    // enough for either form
+    size_t need = orthrus_attend_workspace_bytes(&L);
+    if (need && check_layer(layer) == ORTHRUS_OK && tc_usable(layer) && n_blocks >= 2 &&
+        (long long)n_blocks * layer->block <= (1 << 20)) {
+        const orthrus_layer_t Lp = packed_layer(layer, n_blocks);
+        const size_t n2 = kHeaderBytes + partial_bytes(&Lp, make_plan(&Lp, true), nullptr, true);
+        if (n2 > need) need = n2;
+    }
+    return need;
 }
 
 orthrus_status_t orthrus_multi_block_attend(const orthrus_layer_t *layer, int32_t n_blocks,
@@ -329,6 +394,9 @@ orthrus_status_t orthrus_multi_block_attend(const orthrus_layer_t *layer, int32_
     orthrus_layer_t L;
     if (!anchors || !multi_block_layer(layer, n_blocks, anchors, &L)) return ORTHRUS_ERR_INVALID_ARG;
     if (layer->flags & ORTHRUS_LAYER_BLOCK_IN_CACHE) return ORTHRUS_ERR_INVALID_ARG;
+    if (multi_block_packed(layer, n_blocks))
+        return attend_packed(layer, n_blocks, anchors, q_diff, k_diff_blk, v_diff_blk, out, workspace,
+                             workspace_bytes, stream);
     return attend(&L, 0, q_diff, k_diff_blk, v_diff_blk, out, workspace, workspace_bytes, stream, n_blocks);
 }
 

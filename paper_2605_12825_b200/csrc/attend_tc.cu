@@ -177,7 +177,14 @@ __device__ __noinline__ void merge_tile(int S, int rank, int warp, int lane, int
 
 // Thread r of a softmax warpgroup owns query row r of its tile (TMEM lane r) and all 64 columns of
 // a key tile.  blockIdx.z counts groups of NT query tiles; warpgroup ti works on tile z * NT + ti.
-template <int NT>
+//
+// PACK (multi-block mask, Eq. 6): the p.nb blocks of a sequence, p.kb_width positions each, lie
+// back to back on the position axis (p.K = nb * kb_width), so a 128-row query tile holds the rows
+// of several blocks and the prefix is streamed once for all of them.  Row i belongs to block
+// j = i / kb_width, sees the prefix below its own anchor cache_len[b * nb + j] and the keys of its
+// own block only; the CTA streams up to the largest anchor among the blocks of its query tile,
+// then the 64-key tiles of the block axis that hold those blocks' keys.
+template <int NT, bool PACK>
 __global__ void __launch_bounds__(Shape<NT>::NTHREADS, NT == 1 ? 2 : 1)
 attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const int S, const int kb_rows,
                  const int quiescent)
@@ -244,7 +251,8 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     int b = order / p.Hkv;
     const int h = order % p.Hkv;
     const int len_hi = (int)p.len_cap;
-    if (p.B > 1 && p.B <= 128) {
+    static_assert(!PACK || NT == 1, "the packed form runs one query tile per CTA");
+    if (!PACK && p.B > 1 && p.B <= 128) {
         const int want = b;
         for (int i = tid; i < p.B; i += NTHREADS) {
             const int Pi = min(max(__ldg(p.cache_len + i), 0), len_hi);
@@ -258,20 +266,39 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
         __syncthreads();
         b = *seq_slot;
     }
-    int P = p.cache_len[b];
-    if (P < 0 || P > len_hi) {
-        if (tid == 0 && rank == 0 && p.status) atomicOr(p.status, ORTHRUS_DEV_BAD_CACHE_LEN);
-        P = P < 0 ? 0 : len_hi;
+    int P;
+    int bt_lo = 0, n_blk = 1;               // first tile of block keys on the block axis, how many
+    if constexpr (PACK) {
+        // blocks j_lo..j_hi have rows in this query tile: stream up to their largest anchor
+        const int i0 = tile_i0(0), i1 = min(p.K, i0 + kb_rows) - 1;
+        const int j_lo = i0 / p.kb_width, j_hi = i1 / p.kb_width;
+        bt_lo = j_lo * p.kb_width / TN;
+        n_blk = ((j_hi + 1) * p.kb_width - 1) / TN - bt_lo + 1;
+        P = 0;
+        bool bad = false;
+        for (int j = j_lo; j <= j_hi; ++j) {
+            const int a = __ldg(p.cache_len + (long long)b * p.nb + j);
+            bad |= a < 0 || a > len_hi;
+            P = max(P, min(max(a, 0), len_hi));
+        }
+        if (bad && tid == 0 && rank == 0 && p.status) atomicOr(p.status, ORTHRUS_DEV_BAD_CACHE_LEN);
+    } else {
+        P = p.cache_len[b];
+        if (P < 0 || P > len_hi) {
+            if (tid == 0 && rank == 0 && p.status) atomicOr(p.status, ORTHRUS_DEV_BAD_CACHE_LEN);
+            P = P < 0 ? 0 : len_hi;
+        }
     }
-    // the unit's tiles: n_pre prefix tiles followed by the tile of block keys, shared out evenly
+    // the unit's tiles: n_pre prefix tiles followed by the tile(s) of block keys, shared out evenly
     const uint32_t n_pre = (uint32_t)(P + TN - 1) / TN;
-    const uint32_t t0 = (uint32_t)rank * (n_pre + 1) / (uint32_t)S;
-    const uint32_t t1 = (uint32_t)(rank + 1) * (n_pre + 1) / (uint32_t)S;
+    const uint32_t t0 = (uint32_t)rank * (n_pre + n_blk) / (uint32_t)S;
+    const uint32_t t1 = (uint32_t)(rank + 1) * (n_pre + n_blk) / (uint32_t)S;
     const int n_tiles = (int)(t1 - t0);
-    const bool owner = rank == S - 1;                         // its last tile is the block tile
-    const int n_mine = n_tiles - (owner ? 1 : 0);             // prefix tiles of this CTA
+    // prefix tiles of this CTA; the tiles behind them are block tiles (one, in the last CTA of the
+    // cluster, unless the form is packed)
+    const int n_mine = max(0, min(n_tiles, (int)n_pre - (int)t0));
     const bool active = n_tiles > 0 && aligned;
-    const int row_base = (int)(((long long)(b / p.nb) * p.Hkv + h) * p.capacity);   // row of position 0
+    const int row_base = (int)(((long long)(PACK ? b : b / p.nb) * p.Hkv + h) * p.capacity);   // row of position 0
 
     // The ring holds K and V tiles in the order the MMAs consume them: K0, K1, V0, K2, V1, ...,
     // K(n-1), V(n-2), V(n-1) (the product P.V of a tile is issued after the scores of the next
@@ -292,6 +319,11 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             const int row = row_base + ((int)t0 + t) * TN;
             tma_load_2d(dst, m, 0, row, fb, stream_policy);
             tma_load_2d(dst + SUB_BYTES, m, 64, row, fb, stream_policy);
+        } else if (PACK) {        // tile bt of the block axis: rows >= nb * kb_width arrive as zeros
+            const CUtensorMap *m = is_v ? &tm.vb : &tm.kb;
+            const int bt = bt_lo + (int)t0 + t - (int)n_pre;
+            tma_load_4d(dst, m, 0, h, bt * TN, b, fb);
+            tma_load_4d(dst + SUB_BYTES, m, 64, h, bt * TN, b, fb);
         } else if (p.blk_in_cache) {
             // block tile = the 64 cache rows from P on: rows >= K hold whatever follows the block
             // (masked out of the scores; cleared in the V tile before its product)
@@ -309,7 +341,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
         // the cache rows below cache_len are not being written by the preceding kernel:
         // request the first prefix tiles before waiting for it
         if (active && warp == C::PRODUCER_WARP && lane == 0)
-            while (produced < (owner ? item_of_k(n_tiles - 1) : 2 * n_tiles) && produced < NSLOT) {
+            while (produced < (n_mine < n_tiles ? item_of_k(n_mine) : 2 * n_tiles) && produced < NSLOT) {
                 issue_item(produced); ++produced;     // (stops before the block tile's first item)
             }
         griddep_wait();
@@ -327,6 +359,14 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
         const uint32_t TM_O = C::tm_o(ti);
         float m_run = -INFINITY, l_run = 0.f;
         bool have_o = false;
+        int a_row = 0, k0_row = 0;          // packed form: this row's anchor, first key of its block
+        if constexpr (PACK) {
+            if (valid) {
+                const int j_row = i_row / p.kb_width;
+                a_row = min(max(__ldg(p.cache_len + (long long)b * p.nb + j_row), 0), len_hi);
+                k0_row = j_row * p.kb_width;
+            }
+        }
         if (active && warp_active) {
             // -------------------------------------------------------------- softmax
             const float sc = p.scale_log2;
@@ -342,13 +382,24 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
 #pragma unroll
                 for (int c = 0; c < W / 32; ++c) tmem_ld32(lane_base + TM_S + c * 32, s + c * 32);
                 tmem_ld_wait();
-                // visible columns of this row in this tile
-                int lim;
-                if (t < n_mine) lim = min(TN, P - ((int)t0 + t) * TN);
-                else lim = p.causal ? min(p.K, i_row + 1) : p.K;
+                // visible columns of this row in this tile: [lo, lim)
+                int lim, lo = 0;
+                if constexpr (PACK) {
+                    if (t < n_mine) {
+                        lim = min(TN, a_row - ((int)t0 + t) * TN);
+                    } else {
+                        const int c0 = k0_row - (bt_lo + (int)t0 + t - (int)n_pre) * TN;
+                        lo = max(c0, 0);
+                        lim = min(TN, c0 + p.kb_width);
+                    }
+                    if (lim <= lo) { lim = 0; lo = 0; }
+                } else {
+                    if (t < n_mine) lim = min(TN, P - ((int)t0 + t) * TN);
+                    else lim = p.causal ? min(p.K, i_row + 1) : p.K;
+                }
                 lim = valid ? lim : 0;
                 float mx;
-                if (lim == W) {
+                if (lim == W && lo == 0) {
                     float m4[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q)
@@ -366,9 +417,9 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                     mx = -INFINITY;
 #pragma unroll
                     for (int c = 0; c < W; c += 16) {
-                        if (c < lim) {
+                        if (c < lim && c + 16 > lo) {
 #pragma unroll
-                            for (int j = c; j < c + 16; ++j) if (j < lim) mx = fmaxf(mx, __uint_as_float(s[j]));
+                            for (int j = c; j < c + 16; ++j) if (j < lim && j >= lo) mx = fmaxf(mx, __uint_as_float(s[j]));
                         }
                     }
                 }
@@ -397,7 +448,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                 const float2 nm2 = make_float2(neg_m, neg_m);
                 uint32_t pk[W / 2];                            // this thread's probabilities, packed bf16
                 float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-                if (lim == W) {
+                if (lim == W && lo == 0) {
 #pragma unroll
                     for (int j = 0; j < W; j += 4) {
                         float2 a = __ffma2_rn(make_float2(__uint_as_float(s[j]), __uint_as_float(s[j + 1])), sc2, nm2);
@@ -411,13 +462,13 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                 } else {
 #pragma unroll
                     for (int c = 0; c < W; c += 16) {
-                        if (c < lim) {
+                        if (c < lim && c + 16 > lo) {
 #pragma unroll
                             for (int j = c; j < c + 16; j += 2) {
                                 float p0 = ex2(fmaf(__uint_as_float(s[j]), sc, neg_m));
                                 float p1 = ex2(fmaf(__uint_as_float(s[j + 1]), sc, neg_m));
-                                if (j >= lim) p0 = 0.f;
-                                if (j + 1 >= lim) p1 = 0.f;
+                                if (j >= lim || j < lo) p0 = 0.f;
+                                if (j + 1 >= lim || j + 1 < lo) p1 = 0.f;
                                 acc0.x += p0; acc0.y += p1;
                                 pk[j >> 1] = pack_bf16(p0, p1);
                             }
@@ -747,7 +798,7 @@ int tc_ctas_per_sm(int nt)
 
 namespace {
 
-template <int NT>
+template <int NT, bool PACK = false>
 cudaError_t configure_kernel()
 {   // function attributes belong to a device: set them once on each device that launches
     constexpr int kMaxDevices = 64;
@@ -759,9 +810,9 @@ cudaError_t configure_kernel()
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     std::lock_guard<std::mutex> lock(mu);
     if (!configured[dev]) {
-        e = cudaFuncSetAttribute(attend_tc_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, Shape<NT>::SMEM_BYTES);
+        e = cudaFuncSetAttribute(attend_tc_kernel<NT, PACK>, cudaFuncAttributeMaxDynamicSharedMemorySize, Shape<NT>::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attend_tc_kernel<NT>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            e = cudaFuncSetAttribute(attend_tc_kernel<NT, PACK>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -790,7 +841,7 @@ int max_cluster_of_shape()
             attr[0].val.clusterDim.x = s; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
             cfg.attrs = attr; cfg.numAttrs = 1;
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, attend_tc_kernel<NT>, &cfg) == cudaSuccess && n > 0) { best = s; break; }
+            if (cudaOccupancyMaxActiveClusters(&n, attend_tc_kernel<NT, false>, &cfg) == cudaSuccess && n > 0) { best = s; break; }
             best = s >> 1;
         }
         if (best < 1) best = 1;
@@ -809,11 +860,11 @@ int max_cluster_of_shape()
 int tc_max_cluster(int nt) { return nt == 2 ? max_cluster_of_shape<2>() : max_cluster_of_shape<1>(); }
 int tc_tile_positions() { return TN; }
 
-template <int NT>
+template <int NT, bool PACK = false>
 static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int flags, cudaStream_t st)
 {
     const int S = p.n_splits;
-    cudaError_t e = configure_kernel<NT>();
+    cudaError_t e = configure_kernel<NT, PACK>();
     if (e != cudaSuccess) return e;
     const int row_tiles = (p.K + kb - 1) / kb;
     cudaLaunchConfig_t cfg = {};
@@ -837,7 +888,7 @@ static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int 
     }
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
-    e = cudaLaunchKernelEx(&cfg, attend_tc_kernel<NT>, p, tm, S, kb, (flags & ORTHRUS_LAYER_CACHE_QUIESCENT) ? 1 : 0);
+    e = cudaLaunchKernelEx(&cfg, attend_tc_kernel<NT, PACK>, p, tm, S, kb, (flags & ORTHRUS_LAYER_CACHE_QUIESCENT) ? 1 : 0);
     count_launch();
     return e;
 }
@@ -918,6 +969,20 @@ cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st)
         return cudaErrorInvalidValue;
     }
     return tc_tiles_per_cta(p.G, p.K) == 2 ? launch_tc<2>(p, tm, kb, flags, st) : launch_tc<1>(p, tm, kb, flags, st);
+}
+
+// Packed multi-block form: p.B sequences, p.nb blocks of p.kb_width positions each on one position
+// axis of p.K = nb * kb_width, anchors in p.cache_len[B][nb].
+cudaError_t launch_attend_tc_packed(const AttnParams &p, int flags, cudaStream_t st)
+{
+    const int kb = tc_kb_rows(p.G, p.K);
+    TcMaps tm;
+    const unsigned long long rows = (unsigned long long)p.B * p.Hkv * p.capacity;
+    if (!get_map(p.k_cache, rows, 0, 0, TN, 0, &tm.k) || !get_map(p.v_cache, rows, 0, 0, TN, 0, &tm.v) ||
+        !get_map(p.q, p.Hq, p.K, p.B, p.G, kb, &tm.q) ||
+        !get_map(p.k_blk, p.Hkv, p.K, p.B, 1, TN, &tm.kb) || !get_map(p.v_blk, p.Hkv, p.K, p.B, 1, TN, &tm.vb))
+        return cudaErrorInvalidValue;
+    return launch_tc<1, true>(p, tm, kb, flags, st);
 }
 
 }  // namespace orthrus

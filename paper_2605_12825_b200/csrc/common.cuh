@@ -35,8 +35,9 @@ struct AttnParams {
     int blk_in_cache;   // the block's K/V rows are the cache rows [P, P + K) (k_blk / v_blk unused)
     int nb;             // blocks per sequence: batch entry b reads the cache of sequence b / nb
                         // (1 except for the multi-block mask of Eq. 6, where B counts blocks)
-    long long len_cap;  // largest admissible prefix length (capacity - K; capacity for Eq. 6,
-                        // whose blocks are never stored behind their prefix)
+    int kb_width;       // packed form of Eq. 6 (0 otherwise): B counts sequences, K = nb * kb_width
+                        // positions hold the nb blocks back to back, cache_len is [B][nb]
+    long long len_cap;  // largest admissible prefix length: capacity - block width
     float scale_log2;   // softmax scale times log2(e)
 };
 
@@ -72,6 +73,7 @@ cudaError_t launch_attend_mma(const AttnParams &p, cudaStream_t st);
 int mma_tile_positions();
 bool tc_driver_ok();                    // the driver offers cuTensorMapEncodeTiled
 cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st);   // n_splits = cluster size
+cudaError_t launch_attend_tc_packed(const AttnParams &p, int flags, cudaStream_t st);   // p.kb_width > 0
 int tc_row_tiles(int G, int K);          // 128-row query tiles per unit (0: group too wide)
 int tc_tiles_per_cta(int G, int K);      // query tiles that share one K/V ring in a CTA (1 or 2)
 int tc_cta_groups(int G, int K);         // CTAs along the query-tile axis: ceil(row tiles / tiles per CTA)

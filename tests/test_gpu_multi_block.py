@@ -65,6 +65,59 @@ def test_multi_block_attention_matches_the_oracle(path, shape, splits):
     assert_close(out.t.cpu(), ref, dtype, str(shape))
 
 
+# Shapes of the tcgen05 path whose blocks share query tiles: (S, NB, K, Hq, Hkv, d, L_max)
+PACKED_SHAPES = [
+    (2, 12, 8, 8, 2, 128, 900),     # 3 query tiles of 4 blocks; the third reads tile 1 of the block axis
+    (1, 5, 24, 4, 2, 128, 700),     # blocks straddle query tiles and 64-key tiles of the block axis
+    (2, 7, 16, 2, 2, 128, 500),     # one head per group: 128 positions per query tile, ragged last tile
+    (1, 16, 4, 16, 2, 128, 2500),   # 4-wide blocks, 8 heads per group: 4 blocks per tile
+    (3, 2, 32, 2, 1, 128, 300),     # two blocks fill a tile exactly
+]
+
+
+@pytest.mark.parametrize("shape", PACKED_SHAPES)
+@pytest.mark.parametrize("splits", [0, 1, 4])
+@pytest.mark.parametrize("anchor_mode", ["random", "sorted", "zero"])
+def test_multi_block_packed_query_tiles(shape, splits, anchor_mode):
+    """Blocks that share a 128-row query tile: per-row prefix limits, block-diagonal block keys, block
+    keys spread over several 64-key tiles, clusters with more CTAs than tiles (all anchors 0)."""
+    b = binding()
+    S, NB, K, Hq, Hkv, d, L_max = shape
+    dtype = torch.bfloat16
+    c = make_case(S, NB, K, Hq, Hkv, d, L_max, dtype, seed=sum(shape) + 1)
+    if anchor_mode == "sorted":
+        c["anchors"] = c["anchors"].sort(dim=1).values.contiguous()
+    elif anchor_mode == "zero":
+        c["anchors"].zero_()
+    ref = oracle.multi_block_attend(c["q"], c["k_blk"], c["v_blk"], c["k_cache"], c["v_cache"], c["cache_len"],
+                                    c["anchors"])
+    dev = {k: v.cuda() for k, v in c.items()}
+    # (with every anchor at 0 the bound stays at L_max: clusters larger than the tile count)
+    hint = L_max if anchor_mode == "zero" else int(c["anchors"].max())
+    layer = b.make_layer(dev["k_cache"], dev["v_cache"], dev["cache_len"], Hq, K, hint)
+    outs = {}
+    saved = {k: os.environ.pop(k, None) for k in ("ORTHRUS_SPLITS", "ORTHRUS_MULTI_BLOCK_PACK")}
+    try:
+        if splits:
+            os.environ["ORTHRUS_SPLITS"] = str(splits)
+        for pack in ("1", "0"):
+            os.environ["ORTHRUS_MULTI_BLOCK_PACK"] = pack
+            ws = b.new_workspace(b.orthrus_multi_block_workspace_bytes(layer, NB))
+            out = Guarded(tuple(c["q"].shape), dtype)
+            b.orthrus_multi_block_attend(layer, dev["anchors"], dev["q"], dev["k_blk"], dev["v_blk"], out.t, ws)
+            assert b.orthrus_last_path() == "tcgen05"
+            assert b.orthrus_read_status(ws) == 0
+            assert out.intact()
+            outs[pack] = out.t.cpu()
+    finally:
+        for k, v in saved.items():
+            os.environ.pop(k, None)
+            if v is not None:
+                os.environ[k] = v
+    assert_close(outs["1"], ref, dtype, f"packed {shape}")
+    assert_close(outs["0"], ref, dtype, f"one unit per block {shape}")
+
+
 def test_multi_block_fp32_mode_and_single_block_case():
     """fp32 test mode at 1e-5; and one block per sequence anchored at the clean length gives the very
     bytes orthrus_diffusion_block_attend gives (the same launch on the same data)."""
