@@ -63,7 +63,7 @@ def measured_tensor_peak():
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/, each
 # with the first 16 hex digits of the SHA-256 of the kernel sources the capture was taken
 # from: once those files change the figure is stale and None is reported.
-NCU_TRAFFIC = {"cfg2_8b_b1": (17052416, "d742885a680802a2")}
+NCU_TRAFFIC = {"cfg2_8b_b1": (17052416, "dad9134ecad8fd4d")}
 NCU_TRAFFIC_SOURCES = ("attend_tc.cu", "tc_ptx.cuh")
 NCU_TRAFFIC_LM_HEAD = {("cfg2_8b_b1", 4096): (1249568280, "5112ef6ba5d70c0f"),
                        ("cfg3_ragged", 4096): (1067102904, "5112ef6ba5d70c0f")}
@@ -714,6 +714,16 @@ def run_gpu(args):
         dist.barrier()
     from paper_2605_12825_b200 import binding as B
 
+    if args.multi_block_only:
+        # the multi-block call alone (for profiles): its own small line, not the benchmark's
+        stream = torch.cuda.Stream(device=dev)
+        with torch.cuda.stream(stream):
+            res = multi_block_entry(B, dev, stream, reps=max(1, min(args.steps, 20)))
+        if rank == 0:
+            print(json.dumps({"multi_block_eq6": res}), flush=True)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     wl = W.CONFIGS[args.workload]
     if args.block:
         wl = wl.with_(block=args.block, name=f"{wl.name}_K{args.block}")
@@ -1218,6 +1228,8 @@ def main():
     ap.add_argument("--no-early-launch", action="store_true",
                     help="launch the attention kernels in plain stream order")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--multi-block-only", action="store_true",
+                    help="only the multi-block (Eq. 6) call of the key multi_block_eq6, for profiles")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     args = ap.parse_args()
     if args.impl == "reference":

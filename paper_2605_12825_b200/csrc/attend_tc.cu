@@ -206,7 +206,10 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     const int order = blockIdx.y;
     // query tile ti of this CTA: kb_rows block positions x G heads (at most 128 rows); the last
     // group of a unit may hold fewer than NT tiles
-    auto tile_i0 = [&](int ti) { return ((int)blockIdx.z * NT + ti) * kb_rows; };
+    // (packed form: anchors usually grow along a sequence, so the last query tiles, which stream the
+    //  longest prefixes, are handed out first)
+    const int zt = PACK ? (int)(gridDim.z - 1 - blockIdx.z) : (int)blockIdx.z;
+    auto tile_i0 = [&](int ti) { return (zt * NT + ti) * kb_rows; };
     auto tile_rows = [&](int ti) { return max(0, min(p.K - tile_i0(ti), kb_rows)) * p.G; };
     const bool aligned = (sbase & 1023u) == 0;                // swizzled tiles need 1 KB alignment
 
