@@ -631,6 +631,27 @@ def workload_entry(B, name, dev, stream, flags, steps, gpu_index, peak, min_regi
     st.free()
     del tw, st
     torch.cuda.empty_cache()
+    if wl.layers < 4:
+        # The same calls as a model chains them: four layers with tensors of their own, so every
+        # attention phase is four calls back to back in one graph, each placed (and its first tiles
+        # requested) while its predecessor finishes.  A single call per graph launch, as above, also
+        # pays the launch of its graph inside the events that bracket it.
+        tw = TimedWorkload(B, wl, 4, dev, stream, flags)
+        chained = {"layers": 4}
+        for key, region in (("burst", 0.0), ("sustained", min_region_s)):
+            r4 = tw.run_timed(steps, 3, region, gpu_index)
+            us = (r4["phase_ms"][0] + r4["phase_ms"][1]) / 8 * 1e3
+            chained[key] = {"achieved": round(call_bytes / (us * 1e-6) / 1e9, 2), "peak": peak, "unit": "GB/s",
+                            "frac": round(call_bytes / (us * 1e-6) / 1e9 / peak, 4), "avg_launch_us": round(us, 3),
+                            "inner_repeats": r4["inner"],
+                            "clocks": {k: r4["clocks"].get(k) for k in ("sm_mhz", "samples", "reasons")}}
+        if B.orthrus_read_status(tw.st.ws, stream) != 0:
+            raise SystemExit(f"bench.py: {name}: device status word set after the chained region")
+        out["roofline_chained_layers"] = chained
+        tw.graphs = None
+        tw.st.free()
+        del tw
+        torch.cuda.empty_cache()
     return out
 
 
