@@ -17,6 +17,8 @@
 //              the MMAs consume them.
 //   warp 5     TMEM allocation and MMA issue: S = Q.K^T into one of two score buffers
 //              (so that QK(t+1) runs under softmax(t)), then O += P.V.
+// Units of at most 64 rows run a variant of this CTA (see the kernel's comment): probabilities
+// through shared memory, the two products issued by two warps.
 // The output accumulator O stays in TMEM for the whole CTA.  The running max is only
 // raised when a tile exceeds it by more than 2^8; then, and only then, the owner threads
 // rescale their O rows in TMEM.  Probabilities are bounded by 2^8, which fp32 sums and
@@ -87,7 +89,10 @@ template <int NT> struct Shape {
     static constexpr int BAR_PFULL = BAR_SFULL + 2 * NT;       // + ti * 2 + buffer
     static constexpr int BAR_PVDONE = BAR_PFULL + 2 * NT;      // + ti
     static constexpr int BAR_ALLDONE = BAR_PVDONE + NT;        // + ti
-    static constexpr int NUM_BARS = BAR_ALLDONE + NT;
+    // small-row form of the narrow shape: "scores of buffer b read" and "P buffer b consumed"
+    static constexpr int BAR_SREAD = BAR_ALLDONE + NT;         // + buffer
+    static constexpr int BAR_PFREE = BAR_SREAD + 2;            // + buffer
+    static constexpr int NUM_BARS = BAR_PFREE + 2;
     static_assert(NUM_BARS <= MAX_BARS, "barrier area");
     // TMEM columns: the NT output accumulators, then two score buffers per query tile
     static constexpr uint32_t TM_COLS = 256 * NT;
@@ -156,9 +161,9 @@ __device__ inline void l2_merge_tasks(int S, int rank, int warp, int lane, int n
 // per lane) do not add to those of the streaming loop.  out_tile: the output row of the tile's
 // first block position and first head of the group; row R = i * G + g lies (i * Hq + g) rows on.
 template <int LOADS>
-__device__ __noinline__ void merge_tile(int S, int rank, int warp, int lane, int n_warps, int rows_here,
-                                        const float4 *grp_o, const float2 *grp_ml, __nv_bfloat16 *out_tile,
-                                        int G, int Hq)
+__device__ __forceinline__ void merge_tile_body(int S, int rank, int warp, int lane, int n_warps, int rows_here,
+                                                const float4 *grp_o, const float2 *grp_ml, __nv_bfloat16 *out_tile,
+                                                int G, int Hq)
 {
     const int n_tasks = ((rows_here + 31) >> 5) * (HD / 4);
     auto run = [&](auto sp) {
@@ -174,6 +179,13 @@ __device__ __noinline__ void merge_tile(int S, int rank, int warp, int lane, int
     else if (S <= 8) run(std::integral_constant<int, 8>());
     else run(std::integral_constant<int, 16>());
 }
+template <int LOADS>
+__device__ __noinline__ void merge_tile(int S, int rank, int warp, int lane, int n_warps, int rows_here,
+                                        const float4 *grp_o, const float2 *grp_ml, __nv_bfloat16 *out_tile,
+                                        int G, int Hq)
+{
+    merge_tile_body<LOADS>(S, rank, warp, lane, n_warps, rows_here, grp_o, grp_ml, out_tile, G, Hq);
+}
 
 // Thread r of a softmax warpgroup owns query row r of its tile (TMEM lane r) and all 64 columns of
 // a key tile.  blockIdx.z counts groups of NT query tiles; warpgroup ti works on tile z * NT + ti.
@@ -184,14 +196,23 @@ __device__ __noinline__ void merge_tile(int S, int rank, int warp, int lane, int
 // j = i / kb_width, sees the prefix below its own anchor cache_len[b * nb + j] and the keys of its
 // own block only; the CTA streams up to the largest anchor among the blocks of its query tile,
 // then the 64-key tiles of the block axis that hold those blocks' keys.
-template <int NT, bool PACK>
-__global__ void __launch_bounds__(Shape<NT>::NTHREADS, NT == 1 ? 2 : 1)
+//
+// SM (at most 64 query rows, narrow shape, not packed): the chain score tile -> softmax -> P.V ->
+// next score tile is what a short chunk waits for, and an issuing thread is held about 110 cycles
+// per tcgen05.mma.  Here the probabilities go to shared memory (the unused upper halves of the
+// query tile's two sub-tiles) instead of back into the score buffer, so a score buffer is free
+// again as soon as its softmax threads have read it, and the two products are issued by two
+// warps.  256 threads: warps 0-3 softmax (200 registers after setmaxnreg), 4 producer, 5 Q.K^T,
+// 6 P.V, 7 idle (56 registers).
+template <int NT, bool PACK, bool SM>
+__global__ void __launch_bounds__(SM ? 256 : Shape<NT>::NTHREADS, NT == 1 ? 2 : 1)
 attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const int S, const int kb_rows,
                  const int quiescent)
 {
     using C = Shape<NT>;
     constexpr int W = TN;                     // score columns per softmax thread
-    constexpr int NSLOT = C::NSLOT, NTHREADS = C::NTHREADS;
+    static_assert(!SM || (NT == 1 && !PACK), "the small-row form is a variant of the plain narrow shape");
+    constexpr int NSLOT = C::NSLOT, NTHREADS = SM ? 256 : C::NTHREADS;
     constexpr int OFF_Q = C::OFF_Q, OFF_RING = C::OFF_RING, OFF_BAR = C::OFF_BAR, OFF_MISC = C::OFF_MISC;
     constexpr int BAR_FULL = C::BAR_FULL, BAR_EMPTY = C::BAR_EMPTY, BAR_QFULL = C::BAR_QFULL;
     extern __shared__ __align__(1024) unsigned char smem[];
@@ -231,6 +252,11 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             }
             mbar_init(bar(C::BAR_PVDONE + ti), 1);
             mbar_init(bar(C::BAR_ALLDONE + ti), 1);
+            if constexpr (SM)
+                for (int sb = 0; sb < 2; ++sb) {
+                    mbar_init(bar(C::BAR_SREAD + sb), n_act);
+                    mbar_init(bar(C::BAR_PFREE + sb), 1);
+                }
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
@@ -351,6 +377,11 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     }
     griddep_launch();
 
+    if constexpr (SM) {
+        // the softmax warps take the registers the other four warps do not need
+        if (warp < 4) asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
+        else asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    }
     if (warp < 4 * NT) {
         const int ti = warp >> 2, wq = warp & 3;              // query tile, quarter of its TMEM lanes
         const int r = tid - ti * MROWS;
@@ -385,6 +416,11 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
 #pragma unroll
                 for (int c = 0; c < W / 32; ++c) tmem_ld32(lane_base + TM_S + c * 32, s + c * 32);
                 tmem_ld_wait();
+                if constexpr (SM) {                            // the buffer may take the scores of tile t + 2
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(C::BAR_SREAD + sb));
+                }
                 // visible columns of this row in this tile: [lo, lim)
                 int lim, lo = 0;
                 if constexpr (PACK) {
@@ -482,10 +518,25 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                     }
                 }
                 l_run += (acc0.x + acc0.y) + (acc1.x + acc1.y);
-                // P over the scores, 2 bf16 per 32-bit column
-                tmem_st32(lane_base + TM_S, pk);
-                tmem_st_wait();
-                tc_fence_before();
+                if constexpr (SM) {
+                    // P row r into shared memory buffer sb ([64 rows][64 keys] bf16, 128-byte swizzle),
+                    // once the product of tile t - 2 has read that buffer
+                    if (t >= 2) {
+                        ok = mbar_wait_warp(bar(C::BAR_PFREE + sb), ((t >> 1) - 1) & 1, abort_flag);
+                        if (!ok) break;
+                    }
+                    unsigned char *prow = smem + OFF_Q + (sb ? 3 : 1) * (QSUB_BYTES / 2) + r * 128;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        *reinterpret_cast<uint4 *>(prow + ((c ^ (r & 7)) << 4)) =
+                            make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                    fence_proxy_async();
+                } else {
+                    // P over the scores, 2 bf16 per 32-bit column
+                    tmem_st32(lane_base + TM_S, pk);
+                    tmem_st_wait();
+                    tc_fence_before();
+                }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(C::BAR_PFULL + ti * 2 + sb));
             }
@@ -531,7 +582,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             if (have_o) {
                 // the narrow shape reads the whole row out at once (one wait instead of four), the
                 // wide one, with fewer registers per thread, in two halves; 16-byte stores follow
-                constexpr int PIECE = NT == 1 ? HD : HD / 2;
+                constexpr int PIECE = (NT == 1 && !SM) ? HD : HD / 2;
 #pragma unroll 1
                 for (int c0 = 0; c0 < HD; c0 += PIECE) {
                     uint32_t o[PIECE];
@@ -551,6 +602,22 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
             if (valid) __stcg(my_ml + r, make_float2(have_o ? m_run : -INFINITY, have_o ? l_run : 0.f));
         }
         tc_fence_before();
+        if constexpr (SM) {
+            // These warps hold the registers the merge wants, so they finish the unit here: the
+            // CTA-wide barrier the other warps take below (after it the TMEM is freed), then the
+            // cluster barrier and this CTA's share of the merge.
+            asm volatile("bar.sync 0;" ::: "memory");
+            if (S == 1) return;
+            cluster_sync_all();
+            const int rows_here0 = tile_rows(0);
+            __nv_bfloat16 *out_tile = static_cast<__nv_bfloat16 *>(p.out) +
+                                      (((long long)b * p.K + tile_i0(0)) * p.Hq + h * p.G) * HD;
+            const long long grp_lin = ((long long)blockIdx.z * gridDim.y + order) * S;
+            merge_tile_body<16>(S, rank, warp, lane, 4, rows_here0,
+                                reinterpret_cast<const float4 *>(p.part_o + grp_lin * (MROWS * HD)),
+                                reinterpret_cast<const float2 *>(p.part_ml + grp_lin * (MROWS * 2)), out_tile, p.G, p.Hq);
+            return;
+        }
     } else if (warp == C::PRODUCER_WARP) {
         // ------------------------------------------------------------------ producer
         if (active && lane == 0) {
@@ -581,9 +648,9 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                 mbar_wait(bar(BAR_QFULL), 0, &dummy);
             }
         }
-    } else if (active && tile_rows(warp - C::MMA_WARP) > 0) {
+    } else if (active && (SM ? warp <= C::MMA_WARP + 1 : tile_rows(warp - C::MMA_WARP) > 0)) {
         // ------------------------------------------------------------------ MMA issue, query tile ti
-        const int ti = warp - C::MMA_WARP;
+        const int ti = SM ? 0 : warp - C::MMA_WARP;
         constexpr uint32_t IDESC_QK = make_idesc(TN, 0);      // A = Q, B = K tile, both K-major
         constexpr uint32_t IDESC_PV = make_idesc(HD, 1);      // A = P (TMEM), B = V tile (MN-major)
         const uint32_t q_addr = sbase + OFF_Q + ti * 2 * QSUB_BYTES;
@@ -628,21 +695,47 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                 const uint32_t v_addr = sbase + OFF_RING + slot * SLOT_BYTES;
 #pragma unroll
                 for (int kk = 0; kk < TN / 16; ++kk) {        // 16 key positions per MMA
-                    umma_ts(tmem + C::tm_o(ti), tmem + C::tm_s(ti, t & 1) + kk * 8,
-                            make_desc(v_addr + kk * 2048, SUB_BYTES, 1024), IDESC_PV, (t > 0) || (kk > 0));
+                    if constexpr (SM)
+                        umma_ss(tmem + C::tm_o(ti),
+                                make_desc(sbase + OFF_Q + ((t & 1) ? 3 : 1) * (QSUB_BYTES / 2) + kk * 32, 16, 1024),
+                                make_desc(v_addr + kk * 2048, SUB_BYTES, 1024), IDESC_PV, (t > 0) || (kk > 0));
+                    else
+                        umma_ts(tmem + C::tm_o(ti), tmem + C::tm_s(ti, t & 1) + kk * 8,
+                                make_desc(v_addr + kk * 2048, SUB_BYTES, 1024), IDESC_PV, (t > 0) || (kk > 0));
                 }
                 umma_commit(bar(BAR_EMPTY + slot));
                 umma_commit(bar(C::BAR_PVDONE + ti));
+                if constexpr (SM) umma_commit(bar(C::BAR_PFREE + (t & 1)));
                 if (t == n_tiles - 1) umma_commit(bar(C::BAR_ALLDONE + ti));
             }
             __syncwarp();
             return true;
         };
-        bool ok = mbar_wait_warp(bar(BAR_QFULL), 0, abort_flag);
-        if (ok) { tc_fence_after(); ok = issue_qk(0); }
-        for (int t = 0; t < n_tiles && ok; ++t) {
-            if (t + 1 < n_tiles) ok = issue_qk(t + 1);
-            if (ok) ok = issue_pv(t);
+        bool ok = true;
+        if constexpr (SM) {
+            if (warp == C::MMA_WARP) {
+                // scores of tile t go into buffer t & 1 once the softmax threads of tile t - 2 have
+                // read theirs out of it (one completion of that barrier per use of the buffer, so
+                // the waiter is never more than one phase behind)
+                ok = mbar_wait_warp(bar(BAR_QFULL), 0, abort_flag);
+                if (ok) tc_fence_after();
+                for (int t = 0; t < n_tiles && ok; ++t) {
+                    if (t >= 2) {
+                        ok = mbar_wait_warp(bar(C::BAR_SREAD + (t & 1)), ((t >> 1) - 1) & 1, abort_flag);
+                        if (ok) tc_fence_after();
+                    }
+                    if (ok) ok = issue_qk(t);
+                }
+            } else {
+                for (int t = 0; t < n_tiles && ok; ++t) ok = issue_pv(t);
+            }
+        } else {
+            ok = mbar_wait_warp(bar(BAR_QFULL), 0, abort_flag);
+            if (ok) { tc_fence_after(); ok = issue_qk(0); }
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                if (t + 1 < n_tiles) ok = issue_qk(t + 1);
+                if (ok) ok = issue_pv(t);
+            }
         }
         // every MMA of this warp must have retired before TMEM is freed
         if (ok) mbar_wait_warp(bar(C::BAR_ALLDONE + ti), 0, abort_flag);
@@ -654,21 +747,23 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
     tc_fence_after();
     if (warp == C::MMA_WARP)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::TM_COLS) : "memory");
-    if (tid == 0 && *abort_flag && p.status) atomicOr(p.status, ORTHRUS_DEV_WAIT_TIMEOUT);
+    if (tid == (SM ? 128 : 0) && *abort_flag && p.status) atomicOr(p.status, ORTHRUS_DEV_WAIT_TIMEOUT);
     if (S == 1) return;
     constexpr int NWARPS = NTHREADS / 32;
     // The cluster is what guarantees that the CTAs waiting for one another are resident
     // together.  Release / acquire at cluster scope: every CTA's partial rows are in place.
     cluster_sync_all();
-    for (int ti = 0; ti < NT; ++ti) {
-        const int rows_here = tile_rows(ti);
-        if (rows_here == 0) break;
-        __nv_bfloat16 *out_tile = static_cast<__nv_bfloat16 *>(p.out) +
-                                  (((long long)b * p.K + tile_i0(ti)) * p.Hq + h * p.G) * HD;
-        const long long grp_lin = (((long long)blockIdx.z * NT + ti) * gridDim.y + order) * S;
-        merge_tile<NT == 1 ? 16 : 8>(S, rank, warp, lane, NWARPS, rows_here,
-                   reinterpret_cast<const float4 *>(p.part_o + grp_lin * (MROWS * HD)),
-                   reinterpret_cast<const float2 *>(p.part_ml + grp_lin * (MROWS * 2)), out_tile, p.G, p.Hq);
+    if constexpr (!SM) {                  // (in the small-row form the softmax warps merge; they never come here)
+        for (int ti = 0; ti < NT; ++ti) {
+            const int rows_here = tile_rows(ti);
+            if (rows_here == 0) break;
+            __nv_bfloat16 *out_tile = static_cast<__nv_bfloat16 *>(p.out) +
+                                      (((long long)b * p.K + tile_i0(ti)) * p.Hq + h * p.G) * HD;
+            const long long grp_lin = (((long long)blockIdx.z * NT + ti) * gridDim.y + order) * S;
+            merge_tile<NT == 1 ? 16 : 8>(S, rank, warp, lane, NWARPS, rows_here,
+                       reinterpret_cast<const float4 *>(p.part_o + grp_lin * (MROWS * HD)),
+                       reinterpret_cast<const float2 *>(p.part_ml + grp_lin * (MROWS * 2)), out_tile, p.G, p.Hq);
+        }
     }
 }
 
@@ -801,7 +896,7 @@ int tc_ctas_per_sm(int nt)
 
 namespace {
 
-template <int NT, bool PACK = false>
+template <int NT, bool PACK = false, bool SM = false>
 cudaError_t configure_kernel()
 {   // function attributes belong to a device: set them once on each device that launches
     constexpr int kMaxDevices = 64;
@@ -813,9 +908,9 @@ cudaError_t configure_kernel()
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     std::lock_guard<std::mutex> lock(mu);
     if (!configured[dev]) {
-        e = cudaFuncSetAttribute(attend_tc_kernel<NT, PACK>, cudaFuncAttributeMaxDynamicSharedMemorySize, Shape<NT>::SMEM_BYTES);
+        e = cudaFuncSetAttribute(attend_tc_kernel<NT, PACK, SM>, cudaFuncAttributeMaxDynamicSharedMemorySize, Shape<NT>::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attend_tc_kernel<NT, PACK>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            e = cudaFuncSetAttribute(attend_tc_kernel<NT, PACK, SM>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -844,7 +939,7 @@ int max_cluster_of_shape()
             attr[0].val.clusterDim.x = s; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
             cfg.attrs = attr; cfg.numAttrs = 1;
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, attend_tc_kernel<NT, false>, &cfg) == cudaSuccess && n > 0) { best = s; break; }
+            if (cudaOccupancyMaxActiveClusters(&n, attend_tc_kernel<NT, false, false>, &cfg) == cudaSuccess && n > 0) { best = s; break; }
             best = s >> 1;
         }
         if (best < 1) best = 1;
@@ -863,16 +958,16 @@ int max_cluster_of_shape()
 int tc_max_cluster(int nt) { return nt == 2 ? max_cluster_of_shape<2>() : max_cluster_of_shape<1>(); }
 int tc_tile_positions() { return TN; }
 
-template <int NT, bool PACK = false>
+template <int NT, bool PACK = false, bool SM = false>
 static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int flags, cudaStream_t st)
 {
     const int S = p.n_splits;
-    cudaError_t e = configure_kernel<NT, PACK>();
+    cudaError_t e = configure_kernel<NT, PACK, SM>();
     if (e != cudaSuccess) return e;
     const int row_tiles = (p.K + kb - 1) / kb;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(S, p.B * p.Hkv, (row_tiles + NT - 1) / NT);
-    cfg.blockDim = dim3(Shape<NT>::NTHREADS);
+    cfg.blockDim = dim3(SM ? 256 : Shape<NT>::NTHREADS);
     cfg.dynamicSmemBytes = Shape<NT>::SMEM_BYTES;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
@@ -891,7 +986,7 @@ static cudaError_t launch_tc(const AttnParams &p, const TcMaps &tm, int kb, int 
     }
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
-    e = cudaLaunchKernelEx(&cfg, attend_tc_kernel<NT, PACK>, p, tm, S, kb, (flags & ORTHRUS_LAYER_CACHE_QUIESCENT) ? 1 : 0);
+    e = cudaLaunchKernelEx(&cfg, attend_tc_kernel<NT, PACK, SM>, p, tm, S, kb, (flags & ORTHRUS_LAYER_CACHE_QUIESCENT) ? 1 : 0);
     count_launch();
     return e;
 }
@@ -971,7 +1066,12 @@ cudaError_t launch_attend_tc(const AttnParams &p, int flags, cudaStream_t st)
     } else if (!get_map(p.k_blk, p.Hkv, p.K, p.B, 1, TN, &tm.kb) || !get_map(p.v_blk, p.Hkv, p.K, p.B, 1, TN, &tm.vb)) {
         return cudaErrorInvalidValue;
     }
-    return tc_tiles_per_cta(p.G, p.K) == 2 ? launch_tc<2>(p, tm, kb, flags, st) : launch_tc<1>(p, tm, kb, flags, st);
+    if (tc_tiles_per_cta(p.G, p.K) == 2) return launch_tc<2>(p, tm, kb, flags, st);
+    // at most 64 query rows: the form with the probabilities in shared memory and two issuing warps
+    // (ORTHRUS_TC_SMALL_ROWS=0 keeps the common form: a measurement knob)
+    static const bool small_rows = [] { const char *e = getenv("ORTHRUS_TC_SMALL_ROWS"); return !(e && e[0] == '0'); }();
+    if (small_rows && p.G * p.K <= MROWS / 2) return launch_tc<1, false, true>(p, tm, kb, flags, st);
+    return launch_tc<1>(p, tm, kb, flags, st);
 }
 
 // Packed multi-block form: p.B sequences, p.nb blocks of p.kb_width positions each on one position

@@ -26,10 +26,17 @@ __device__ inline bool mbar_try(uint32_t bar, uint32_t parity) {
                  " selp.u32 %0, 1, 0, p;\n}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// non-blocking probe of a phase
+__device__ inline bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+                 " selp.u32 %0, 1, 0, p;\n}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait.  Returns false (and raises the CTA's abort flag) if the phase does not
 // complete within about a second, or if another thread already gave up.
 __device__ inline bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    if (mbar_try(bar, parity)) return true;
+    if (mbar_test(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t it = 1; it < (1u << 24); ++it) {
         if (mbar_try(bar, parity)) return true;
