@@ -676,13 +676,18 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
         auto issue_pv = [&](int t) -> bool {
             const int j = item_of_v(t), slot = j % NSLOT;
             if (!mbar_wait_warp(bar(BAR_FULL + slot), (j / NSLOT) & 1, abort_flag)) return false;
-            // a ragged prefix tile: V rows past the prefix may hold anything, and 0 * NaN would
-            // poison the product, so they are cleared before the MMA reads them (by every MMA
-            // warp: the same zeros, and no warp has to wait for another)
-            const int nv = t < n_mine ? min(TN, P - ((int)t0 + t) * TN) : (p.blk_in_cache ? p.K : TN);
-            if (nv < TN) {
+            // Only the 16-key groups that hold keys are multiplied (an instruction costs its issuing
+            // thread the same whatever its size): the block's own tile is K keys wide, a ragged
+            // prefix tile ends at the prefix.  In the last group, V rows past the keys may hold
+            // anything where they come from the cache, and 0 * NaN would poison the product, so
+            // they are cleared before the MMA reads them (by every MMA warp: the same zeros, and
+            // no warp has to wait for another); rows of the block's own tensor past K arrive as zeros.
+            const bool from_cache = t < n_mine || p.blk_in_cache;
+            const int nv = t < n_mine ? min(TN, P - ((int)t0 + t) * TN) : (PACK ? TN : p.K);
+            const int n_kk = (nv + 15) >> 4;
+            if (from_cache && nv < n_kk * 16) {
                 unsigned char *vt = smem + OFF_RING + slot * SLOT_BYTES;
-                for (int e = lane; e < (TN - nv) * 16; e += 32) {
+                for (int e = lane; e < (n_kk * 16 - nv) * 16; e += 32) {
                     const int rr = nv + (e >> 4), c = e & 15;
                     *reinterpret_cast<uint4 *>(vt + sw_off(rr, c, SUB_BYTES)) = make_uint4(0, 0, 0, 0);
                 }
@@ -695,6 +700,7 @@ attend_tc_kernel(const AttnParams p, const __grid_constant__ TcMaps tm, const in
                 const uint32_t v_addr = sbase + OFF_RING + slot * SLOT_BYTES;
 #pragma unroll
                 for (int kk = 0; kk < TN / 16; ++kk) {        // 16 key positions per MMA
+                    if (kk >= n_kk) break;
                     if constexpr (SM)
                         umma_ss(tmem + C::tm_o(ti),
                                 make_desc(sbase + OFF_Q + ((t & 1) ? 3 : 1) * (QSUB_BYTES / 2) + kk * 32, 16, 1024),
